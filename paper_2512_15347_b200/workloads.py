@@ -1,0 +1,188 @@
+"""Seeded synthetic inputs and the five workload shapes.
+
+This module produces *inputs only* (initial latents, stand-in network predictions,
+stand-in reward-model scores, per-step schedule coefficients).  It contains none of the
+rollout arithmetic and imports neither the CUDA binding nor any checker, so the GPU
+library and an independent CPU check can both be fed the very same arrays.
+
+The denoiser, VAE decoder and reward model of the paper are not available; their
+outputs are replaced by seeded random tensors with the shapes of the paper's
+workloads (Stable-Diffusion style 4x32x32 / 4x64x64 latents, SD3 / FLUX style
+16x128x128 latents; group schedules such as 48->24->12 from the experimental
+settings of Section 6.1).
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass
+from typing import Dict, List, Optional, Tuple
+
+import numpy as np
+import torch
+
+
+@dataclass(frozen=True)
+class Workload:
+    name: str
+    n_groups: int                 # G prompt groups
+    n_expand: int                 # N0 = G_max trajectories per group
+    stages: Tuple[Tuple[int, int], ...]   # (step index, survivors per group)
+    n_steps: int                  # T
+    elems: int                    # d = C*H*W
+    channels: int
+    vel_dtype: str                # "fp32" | "bf16"
+    seed: int
+    velocity: str                 # "affine" (config 1) | "normal" (fresh N(0,1) per step)
+    scores: str                   # "preview" | "external"
+    sigma: float = 0.7            # noise_std = sigma * sqrt(dt)
+    adv_eps: float = 1e-6
+
+    @property
+    def final_keep(self) -> int:
+        return self.stages[-1][1] if self.stages else self.n_expand
+
+    def active_at(self, step: int) -> int:
+        """Trajectories per group that take SDE step `step` (pruning precedes the step)."""
+        k = self.n_expand
+        for s, keep in self.stages:
+            if step >= s:
+                k = keep
+        return k
+
+    def rows_before(self, step: int) -> int:
+        """Trajectories per group alive when the prediction for `step` is made."""
+        k = self.n_expand
+        for s, keep in self.stages:
+            if step > s:
+                k = keep
+        return k
+
+    @property
+    def traj_steps(self) -> int:
+        return sum(self.n_groups * self.active_at(s) for s in range(self.n_steps))
+
+    @property
+    def element_steps(self) -> int:
+        return self.traj_steps * self.elems
+
+    @property
+    def score_rows(self) -> int:
+        """Rows scored from (x, v) over all stages (0 for external scores)."""
+        if self.scores != "preview":
+            return 0
+        return sum(self.n_groups * self.rows_before(s) for s, _ in self.stages)
+
+    def step_coef(self, step: int) -> Tuple[float, float, float]:
+        """(c_x, c_v, noise_std): drift = the supplied prediction, uniform dt = 1/T."""
+        dt = 1.0 / self.n_steps
+        return 1.0, dt, self.sigma * math.sqrt(dt)
+
+    def preview_coef(self, step: int) -> Tuple[float, float]:
+        """(p_x, p_v): one Euler step of the probability-flow ODE over the remaining time."""
+        return 1.0, 1.0 - step / self.n_steps
+
+
+WORKLOADS: Dict[str, Workload] = {
+    "tiny": Workload("tiny", 1, 16, ((3, 8),), 10, 4 * 32 * 32, 4, "fp32", 0, "affine", "preview"),
+    "sd15": Workload("sd15", 8, 24, ((4, 12),), 20, 4 * 64 * 64, 4, "bf16", 1, "normal", "preview"),
+    "sd3": Workload("sd3", 16, 48, ((3, 24), (6, 12)), 28, 16 * 128 * 128, 16, "bf16", 3,
+                    "normal", "external"),
+    "large": Workload("large", 64, 64, ((2, 32), (5, 16), (8, 16)), 28, 16 * 128 * 128, 16, "bf16",
+                      7, "normal", "preview"),
+}
+
+# OVF selection microbenchmark: 4096 groups x 256 scores, keep 32.
+OVF_MICRO = dict(n_groups=4096, n=256, k=32, seed=4)
+
+
+def scaled(w: Workload, *, n_groups: Optional[int] = None, elems: Optional[int] = None,
+           name: Optional[str] = None) -> Workload:
+    """A smaller copy of a workload (fewer groups and/or shorter latents) for quick checks."""
+    from dataclasses import replace
+    return replace(w, n_groups=n_groups or w.n_groups, elems=elems or w.elems,
+                   name=name or (w.name + "-scaled"))
+
+
+def _gen(device, *words: int) -> torch.Generator:
+    g = torch.Generator(device=device)
+    s = 0x9E3779B97F4A7C15
+    for w in words:
+        s = (s ^ (int(w) + 0x632BE59BD9B4E019)) * 0xD1342543DE82EF95 % (1 << 63)
+    g.manual_seed(s)
+    return g
+
+
+def initial_latents(w: Workload, device="cpu") -> torch.Tensor:
+    """x_0 ~ N(0, I), fp32 [G*N0, d]."""
+    return torch.randn(w.n_groups * w.n_expand, w.elems, generator=_gen(device, w.seed, 101),
+                       device=device, dtype=torch.float32)
+
+
+def normal_velocity(w: Workload, step: int, rows: int, device="cpu") -> torch.Tensor:
+    """Stand-in network prediction for one step: fresh N(0,1), in the workload's dtype."""
+    v = torch.randn(rows, w.elems, generator=_gen(device, w.seed, 202, step), device=device,
+                    dtype=torch.float32)
+    return v.to(torch.bfloat16) if w.vel_dtype == "bf16" else v
+
+
+def affine_field(w: Workload, device="cpu") -> Tuple[torch.Tensor, torch.Tensor]:
+    """Per-channel (a_c, b_c) with a_c ~ U(-1, 0), b_c ~ N(0, 0.1^2), expanded to [d]."""
+    g = _gen("cpu", w.seed, 303)
+    a = -torch.rand(w.channels, generator=g, dtype=torch.float32)
+    b = 0.1 * torch.randn(w.channels, generator=g, dtype=torch.float32)
+    per = w.elems // w.channels
+    return (a.repeat_interleave(per).to(device), b.repeat_interleave(per).to(device))
+
+
+def affine_velocity(x: torch.Tensor, a: torch.Tensor, b: torch.Tensor) -> torch.Tensor:
+    """v = a_c * x + b_c as two separately rounded fp32 operations (identical on CPU and GPU)."""
+    v = x * a
+    v += b
+    return v
+
+
+def _student_t(rng: np.random.Generator, nu: float, size) -> np.ndarray:
+    return rng.standard_t(nu, size=size)
+
+
+def clustered_scores(n_groups: int, n: int, seed: int, stage: int, *, cluster_sigma: float,
+                     outlier_frac: float, outlier_scale: float, nu: float) -> np.ndarray:
+    """Reward-clustered stand-in scores, fp32 [G, n].
+
+    Each group has a mean mu_g ~ U(0,1); a score is mu_g + cluster_sigma*z with probability
+    1 - outlier_frac and mu_g + outlier_scale*t_nu otherwise (heavy-tailed outliers).
+    """
+    rng = np.random.Generator(np.random.Philox(key=[seed, 1000 + stage]))
+    mu = rng.random((n_groups, 1))
+    z = rng.standard_normal((n_groups, n))
+    t = _student_t(rng, nu, (n_groups, n))
+    outlier = rng.random((n_groups, n)) < outlier_frac
+    return (mu + np.where(outlier, outlier_scale * t, cluster_sigma * z)).astype(np.float32)
+
+
+def sd3_stage_scores(w: Workload, stage: int, traj_id: np.ndarray) -> np.ndarray:
+    """External scores for the SD3-shaped workload, keyed by original trajectory and stage.
+
+    A full [G, N0] table is drawn per stage; the entries of the still-active trajectories
+    are returned in their current (compacted) order.
+    """
+    table = clustered_scores(w.n_groups, w.n_expand, w.seed, stage, cluster_sigma=0.05,
+                             outlier_frac=0.15, outlier_scale=0.3, nu=3.0).reshape(-1)
+    return table[np.asarray(traj_id, dtype=np.int64)]
+
+
+def ovf_micro_scores(n_groups: int = OVF_MICRO["n_groups"], n: int = OVF_MICRO["n"],
+                     seed: int = OVF_MICRO["seed"]) -> np.ndarray:
+    """Scores of the OVF microbenchmark: 80 % N(mu_g, 0.02), 20 % Student-t(2) scaled 0.3."""
+    return clustered_scores(n_groups, n, seed, 0, cluster_sigma=0.02, outlier_frac=0.2,
+                            outlier_scale=0.3, nu=2.0)
+
+
+def bf16_bits(t: torch.Tensor) -> np.ndarray:
+    """bf16 tensor (CPU) -> numpy uint16 bit patterns."""
+    return t.contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+def as_numpy_velocity(v: torch.Tensor) -> np.ndarray:
+    v = v.detach().cpu()
+    return bf16_bits(v) if v.dtype == torch.bfloat16 else v.numpy()
