@@ -1,0 +1,245 @@
+/*
+ * progrpo.h - C ABI of the B200 (sm_100a) hot path of the Pro-GRPO
+ * Expand-and-Prune rollout.
+ *
+ * The library advances G prompt groups of N0 expanded trajectories in lockstep
+ * through a T-step reverse-time SDE, scores and prunes them at the scheduled
+ * checkpoints with Optimal Variance Filtering (OVF), keeps only survivors in
+ * later steps and finally normalises the survivors' rewards into
+ * group-relative advantages.  The denoiser, VAE decoder and reward model are
+ * outside: their outputs are passed in as tensors.
+ *
+ * Conventions
+ *  - Every function returns 0 (PG_OK) or a negative PG_E* code; nothing aborts
+ *    or throws.  pg_strerror() names a code; pg_last_cuda_error() returns the
+ *    cudaError_t behind the last PG_ECUDA of the calling thread.
+ *  - All tensor pointers are DEVICE pointers owned by the caller, row-major and
+ *    contiguous, 16-byte aligned unless stated otherwise.  The library owns
+ *    only the opaque handle and its small device scratch (trajectory-id map,
+ *    reduction partials, tickets, status word), all released by
+ *    pg_rollout_destroy().  pg_config and the coefficient structs are HOST
+ *    memory, read during the call only.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
+ *    enqueue work and return; none synchronises, except pg_rollout_status()
+ *    and pg_rollout_host().  All calls on one handle must be issued on one
+ *    stream (or be ordered by the caller): the handle's device state is
+ *    updated in stream order.
+ *  - Rows: at any time the n_active = G * K_i live trajectories are the rows
+ *    of the latent tensor, group-major (row = g * K_i + slot).  Step indices
+ *    are 0-based.  A stage (s, k) prunes every group to k survivors BEFORE the
+ *    SDE update of step s, using the prediction made at x_s; pruned
+ *    trajectories take neither step s nor any later step.
+ *  - Noise: standard normals from Philox4x32-10 (Salmon et al., SC'11) with
+ *    key = (seed low, seed high) and counter = (element / 4, step,
+ *    trajectory id, stream id 0); the trajectory id is
+ *    (group_offset + g) * N0 + original slot and survives compaction.  The four
+ *    output words r0..r3 give elements 4q..4q+3 by Box-Muller on 24-bit
+ *    uniforms: u1 = ((r0 >> 8) + 1) / 2^24, u2 = (r1 >> 8) / 2^24,
+ *    xi = sqrt(-2 ln u1) * (cos, sin)(2 pi u2); likewise (r2, r3).
+ */
+#ifndef PROGRPO_H
+#define PROGRPO_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PG_OK          0
+#define PG_EINVAL     (-1)  /* bad argument, shape, alignment or null pointer        */
+#define PG_ESTATE     (-2)  /* call out of sequence for the handle's schedule          */
+#define PG_ECUDA      (-3)  /* a CUDA runtime call failed; see pg_last_cuda_error()    */
+#define PG_ENONFINITE (-4)  /* reported by pg_rollout_status(): non-finite scores seen */
+#define PG_ETIMEOUT   (-5)  /* reported by pg_rollout_status(): a bounded device wait expired */
+#define PG_ENOMEM     (-6)  /* host or device allocation for the handle failed         */
+
+#define PG_VEL_F32  0
+#define PG_VEL_BF16 1
+
+#define PG_MAX_GROUP 1024   /* largest N0 (trajectories per group) the selection kernels take */
+
+typedef struct pg_rollout pg_rollout; /* opaque */
+
+/* Schedule of one rollout batch (Section 5.2, "Expand and Prune"). */
+typedef struct {
+  int32_t n_groups;        /* G  prompt groups handled by this handle                         */
+  int32_t n_expand;        /* N0 = G_max trajectories per group at step 0, 1..PG_MAX_GROUP     */
+  int32_t elems;           /* d  elements per latent (C*H*W), a positive multiple of 4         */
+  int32_t n_steps;         /* T  SDE steps                                                     */
+  int32_t n_stages;        /* I  pruning checkpoints (may be 0)                                */
+  const int32_t *stage_step; /* [I] strictly increasing, 0 <= step < T                         */
+  const int32_t *stage_keep; /* [I] survivors per group, non-increasing, 1 <= keep <= previous  */
+  uint64_t seed;           /* Philox key                                                       */
+  int32_t group_offset;    /* index of this handle's first group in the whole job (multi-GPU
+                              sharding by groups); enters the trajectory id only             */
+  int32_t vel_dtype;       /* PG_VEL_F32 or PG_VEL_BF16: element type of every `vel` tensor    */
+  int32_t logp_mean;       /* 0: log-density summed over elements; 1: divided by d             */
+  float   adv_eps;         /* epsilon of the advantage denominator, >= 0                       */
+} pg_config;
+
+/* x' = c_x * x + c_v * v + noise_std * xi.  For drift b = v: c_x = 1, c_v = dt,
+ * noise_std = sigma_t * sqrt(dt).  Other backbones (the score-corrected drifts
+ * of Eq. "backbone_drifts_method") are affine in (x, prediction) as well and
+ * use other coefficients.  Evaluated in fp32 on the device. */
+typedef struct { double c_x, c_v, noise_std; } pg_step_coef;
+
+/* x_hat = p_x * x + p_v * v  (Eq. "ode_lookahead_method"; rectified flow:
+ * p_x = 1, p_v = remaining time). */
+typedef struct { double p_x, p_v; } pg_preview_coef;
+
+/*
+ * Creates a handle for one batch (Section 5.1 "Initialization"; Section 5.2).
+ * Allocates the handle's device scratch on the current device.  Errors:
+ * PG_EINVAL for an inconsistent schedule, PG_ENOMEM / PG_ECUDA.
+ */
+int pg_rollout_init(const pg_config *cfg, pg_rollout **out);
+
+/* Frees the handle and its scratch.  The caller must have synchronised the
+ * stream the handle was used on.  NULL is accepted. */
+int pg_rollout_destroy(pg_rollout *h);
+
+/* Rewinds the handle to step 0 / stage 0 with all N0 trajectories active
+ * (enqueues the reset of the trajectory-id map on `stream`). */
+int pg_rollout_reset(pg_rollout *h, void *stream);
+
+/*
+ * Synchronises the device and reports the host-side cursor (trajectories
+ * active in total, next step index) and the device status word (bit 0:
+ * non-finite score seen by pg_prune_ovf, bit 1: a bounded wait expired).
+ * Any out pointer may be NULL.  Returns PG_ENONFINITE / PG_ETIMEOUT if the
+ * corresponding bit is set, else PG_OK.
+ */
+int pg_rollout_status(pg_rollout *h, int32_t *n_active, int32_t *next_step, int32_t *device_status);
+
+/*
+ * SDE step with fused Gaussian policy log-probability (Eq. "euler_method"; the
+ * policy pi_theta of Section 5.1 is the Gaussian N(m, noise_std^2 I) that the
+ * step induces).  For each active row i (src = src_rows ? src_rows[i] : i):
+ *     m      = c_x * x_in[src] + c_v * vel[src]
+ *     x_out[i] = m + noise_std * xi(trajectory id of row i, step)
+ *     logp_out[i] = -1/2 * sum_e xi_e^2 - d/2 * ln(2 pi noise_std^2)   (/ d if logp_mean)
+ * x_in  [rows_in, d] fp32, vel [rows_in, d] fp32 or bf16 (cfg.vel_dtype);
+ * src_rows [n_active] int32 or NULL: gather used on the step that follows a
+ * prune, so that survivors need not be moved first (pass pg_prune_ovf's
+ * src_rows output; x_out must then not alias x_in).  Without src_rows, x_out
+ * may equal x_in.  x_out [n_active, d] fp32; logp_out [n_active] fp32.
+ * noise_std == 0 gives the deterministic update and logp_out = 0.
+ * `step` must be the handle's next step, and a stage scheduled at `step` must
+ * already have been pruned (else PG_ESTATE).  Advances the step cursor.
+ */
+int pg_step(pg_rollout *h, int32_t step, const pg_step_coef *coef, const float *x_in,
+            const void *vel, const int32_t *src_rows, float *x_out, float *logp_out, void *stream);
+
+/*
+ * Latent score at a pruning checkpoint (Eq. "ode_lookahead_method", Eq.
+ * "proxy_reward_method").  The preview x_hat = p_x * x + p_v * vel is reduced
+ * to the stand-in proxy reward r = mean_e(x_hat_e) for each of the n_active
+ * rows: scores_out [n_active] fp32.  preview_out (nullable) [n_active, d] fp32
+ * receives x_hat for an external decoder / reward model.  With p_v == 0 `vel`
+ * is not read and may be NULL (used for the final reward stand-in).  Does not
+ * move any cursor; may be called at any time.
+ */
+int pg_score(pg_rollout *h, const pg_preview_coef *coef, const float *x, const void *vel,
+             float *scores_out, float *preview_out, void *stream);
+
+/*
+ * Optimal Variance Filtering for stage `stage` (Eq. "ovf"; Section 5.1): in
+ * every group keeps the k = stage_keep[stage] of the K_i active trajectories
+ * whose scores have maximal population variance.  The maximiser is found
+ * exactly as the best of the k+1 candidates "j lowest and k-j highest" in the
+ * total order (score, slot); -0 == +0; NaN orders above +inf; non-finite
+ * values enter the variance clamped to +-FLT_MAX and set status bit 0.  Among
+ * equal candidates the largest j wins (all-equal scores keep slots 0..k-1).
+ * scores [G*K_i] fp32; keep_idx [G*k] int32: kept slots within the group,
+ * ascending; src_rows (nullable) [G*k] int32: g*K_i + keep_idx, for pg_step /
+ * external gathers; sel_var (nullable) [G] fp32: the selected variance.
+ * `stage` must be the next unpruned stage and its step the next step (else
+ * PG_ESTATE).  Advances the stage cursor, makes n_active = G*k and compacts the
+ * handle's trajectory-id map in stream order.
+ */
+int pg_prune_ovf(pg_rollout *h, int32_t stage, const float *scores, int32_t *keep_idx,
+                 int32_t *src_rows, float *sel_var, void *stream);
+
+/*
+ * Survivor compaction of a caller-side row array after the most recent
+ * pg_prune_ovf (Section 5.1: pruned trajectories "incur no further SDE
+ * steps"): dst row g*k + p = src row g*K_prev + keep_idx[g*k + p]; order and
+ * count are preserved.  row_bytes > 0; rows need only be byte-aligned, 16-byte
+ * aligned rows are moved with 128-bit accesses.  dst must not overlap src.
+ */
+int pg_compact(pg_rollout *h, const int32_t *keep_idx, const void *src, void *dst,
+               size_t row_bytes, void *stream);
+
+/*
+ * Group-relative advantages over the survivors (Eq. "advantage", Eq. "advK"):
+ * mu = mean, sigma = population standard deviation of the K = n_active / G
+ * rewards of a group, adv = (R - mu) / (sigma + adv_eps).  rewards, adv
+ * [G*K] fp32; mean, std (nullable) [G] fp32.
+ */
+int pg_advantages(pg_rollout *h, const float *rewards, float *adv, float *mean, float *std,
+                  void *stream);
+
+/*
+ * Stateless OVF over many groups in one launch: selection as pg_prune_ovf for
+ * n_groups groups of n scores, keeping k; optionally the kept scores and their
+ * group-relative advantages (Eq. "advK" applied to the kept scores) in the
+ * same kernel.  keep_idx [G*k] int32; kept_scores, adv (nullable) [G*k] fp32;
+ * status (nullable) device int32, bit 0 is OR-ed in when a non-finite score is
+ * seen.  1 <= k <= n <= PG_MAX_GROUP.
+ */
+int pg_ovf_select_batched(int32_t n_groups, int32_t n, int32_t k, const float *scores,
+                          int32_t *keep_idx, float *kept_scores, float *adv, float adv_eps,
+                          int32_t *status, void *stream);
+
+/*
+ * Whole rollout from HOST buffers (Section 5.1 + 5.2 end to end): copies x0
+ * and, step by step, the predictions to the device (copies overlap compute on
+ * a second stream), runs score / OVF / step for every step with the preview
+ * mean as score (or host-supplied scores), then the final reward stand-in
+ * (mean of x_T, or host-supplied rewards) and the advantages, and copies the
+ * results back.  Synchronises before returning.
+ *   x0        host [G*N0, d] fp32
+ *   vel_steps host array of T pointers; vel_steps[s] is [rows_s, d] in
+ *             cfg.vel_dtype with rows_s = rows alive when step s is predicted
+ *             (G*K before any prune scheduled at s)
+ *   step_coef [T], preview_coef [I] host arrays
+ *   stage_scores host array of I pointers to fp32 [rows] or NULL (preview mean)
+ *   final_rewards host fp32 [G*K] or NULL (mean of x_T)
+ *   outputs (host, any may be NULL): x_final [G*K, d], logp [T][...] packed
+ *   step after step (sum over s of rows taking step s), keep_idx packed stage
+ *   after stage, adv [G*K], traj_id [G*K].
+ *   workspace: device memory of at least pg_rollout_host_workspace_bytes(cfg).
+ * Host buffers should be pinned for full copy bandwidth.
+ */
+size_t pg_rollout_host_workspace_bytes(const pg_config *cfg);
+int pg_rollout_host(const pg_config *cfg, const pg_step_coef *step_coef,
+                    const pg_preview_coef *preview_coef, const float *x0,
+                    const void *const *vel_steps, const float *const *stage_scores,
+                    const float *final_rewards, float *x_final, float *logp, int32_t *keep_idx,
+                    float *adv, int32_t *traj_id, void *workspace, size_t workspace_bytes);
+
+/* Copies the handle's current trajectory-id map ([n_active] int32, device
+ * memory) to `dst` (device) in stream order. */
+int pg_rollout_traj_ids(pg_rollout *h, int32_t *dst, void *stream);
+
+/* Raw Philox4x32-10 blocks for n (counter, key) pairs: ctr [n,4], key [n,2],
+ * out [n,4] uint32 device arrays.  Exposes the library's generator so that it
+ * can be compared bit for bit with another implementation. */
+int pg_philox_raw(int64_t n, const uint32_t *ctr, const uint32_t *key, uint32_t *out, void *stream);
+
+/* Standard normals exactly as pg_step draws them: out [n_rows, d] fp32 for
+ * trajectory ids traj_id [n_rows] (device) at `step`, stream id `stream_id`. */
+int pg_normal_rows(uint64_t seed, int32_t step, int32_t stream_id, int32_t n_rows, int32_t d,
+                   const int32_t *traj_id, float *out, void *stream);
+
+const char *pg_strerror(int code);
+int pg_last_cuda_error(void);
+/* Number of kernels the library has launched so far from the calling process. */
+uint64_t pg_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PROGRPO_H */

@@ -1,0 +1,147 @@
+// Shared device helpers and launcher declarations of the Pro-GRPO rollout library (sm_100a).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+
+#include "../../include/progrpo.h"
+
+namespace pg {
+
+// ---------------------------------------------------------------- host-side bookkeeping
+void note_launch();                 // counts kernels launched by the library
+int  cuda_fail(cudaError_t e);      // remembers e for pg_last_cuda_error(), returns PG_ECUDA
+
+#define PG_CUDA(call)                                        \
+  do {                                                       \
+    cudaError_t pg_e_ = (call);                              \
+    if (pg_e_ != cudaSuccess) return ::pg::cuda_fail(pg_e_); \
+  } while (0)
+
+#define PG_LAUNCH_CHECK()                                    \
+  do {                                                       \
+    ::pg::note_launch();                                     \
+    cudaError_t pg_e_ = cudaGetLastError();                  \
+    if (pg_e_ != cudaSuccess) return ::pg::cuda_fail(pg_e_); \
+  } while (0)
+
+// ---------------------------------------------------------------- Philox4x32-10
+// Round keys k + r * (0x9E3779B9, 0xBB67AE85), r = 0..9, precomputed on the host so that the
+// device reads them as immediates from the kernel-parameter bank.
+struct PhiloxKeys {
+  uint32_t k0[10];
+  uint32_t k1[10];
+};
+
+inline PhiloxKeys make_philox_keys(uint64_t seed) {
+  PhiloxKeys rk;
+  uint32_t a = (uint32_t)(seed & 0xFFFFFFFFull), b = (uint32_t)(seed >> 32);
+  for (int r = 0; r < 10; ++r) {
+    rk.k0[r] = a;
+    rk.k1[r] = b;
+    a += 0x9E3779B9u;
+    b += 0xBB67AE85u;
+  }
+  return rk;
+}
+
+#ifdef __CUDACC__
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               const PhiloxKeys& rk) {
+#pragma unroll
+  for (int r = 0; r < 10; ++r) {
+    const uint64_t p0 = (uint64_t)0xD2511F53u * (uint64_t)c0;
+    const uint64_t p1 = (uint64_t)0xCD9E8D57u * (uint64_t)c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ rk.k0[r];
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ rk.k1[r];
+    c1 = (uint32_t)p1;
+    c3 = (uint32_t)p0;
+    c0 = n0;
+    c2 = n2;
+  }
+  return make_uint4(c0, c1, c2, c3);
+}
+
+// Two standard normals from two generator words (24-bit uniforms, Box-Muller).
+//   u1 = ((r0 >> 8) + 1) * 2^-24 in (0, 1],  u2 = (r1 >> 8) * 2^-24 in [0, 1)
+//   a = sqrt(-2 ln u1) cos(2 pi u2),  b = sqrt(-2 ln u1) sin(2 pi u2)
+// The logarithm uses the hardware log2 except close to u1 = 1, where its absolute error would
+// dominate the small radius: there -ln(1 - w) is summed as a short series in w = 1 - u1 (exact
+// in fp32).  The angle is shifted by half a turn (cos(t) = -cos(t - pi), same for sin) so that
+// the hardware sine / cosine are evaluated on [-pi, pi), their most accurate range.
+__device__ __forceinline__ void normal_pair(uint32_t r0, uint32_t r1, float& a, float& b) {
+  const float k1 = (float)(r0 >> 8);
+  const float u1 = fmaf(k1, 5.9604644775390625e-8f, 5.9604644775390625e-8f);
+  float neg2ln = -1.3862943611198906f * __log2f(u1);           // -2 ln(u1) = -2 ln2 * log2(u1)
+  const float w = (float)((~r0) >> 8) * 5.9604644775390625e-8f;  // 1 - u1, exact
+  // -2 ln(1 - w) = 2w + w^2 + (2/3) w^3 + (1/2) w^4 + (2/5) w^5 ...
+  float ser = fmaf(w, 0.4f, 0.5f);
+  ser = fmaf(ser, w, 0.66666666666666667f);
+  ser = fmaf(ser, w, 1.0f);
+  ser = fmaf(ser, w, 2.0f);
+  ser *= w;
+  neg2ln = (w < 0.03125f) ? ser : neg2ln;
+  float radius;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(radius) : "f"(neg2ln));
+  const float turn = fmaf((float)(r1 >> 8), 5.9604644775390625e-8f, -0.5f);  // u2 - 1/2, exact
+  float s, c;
+  __sincosf(6.283185307179586f * turn, &s, &c);
+  a = -radius * c;
+  b = -radius * s;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+__device__ __forceinline__ double warp_sum(double v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+#endif  // __CUDACC__
+
+// ---------------------------------------------------------------- launch geometry
+constexpr int kRowThreads = 256;       // threads per CTA of the row-streaming kernels
+constexpr int kQuadsPerThread = 8;     // 4-element quads per thread and CTA
+constexpr int kChunkQuads = kRowThreads * kQuadsPerThread;   // 2048 quads = 8192 elements
+
+inline int chunks_per_row(int elems) { return (elems / 4 + kChunkQuads - 1) / kChunkQuads; }
+
+// ---------------------------------------------------------------- launchers (device pointers)
+struct RowScratch {
+  float* partials;        // [rows * chunks_per_row]
+  unsigned int* tickets;  // [rows], zero between launches
+};
+
+int launch_step(int n_rows, int elems, int vel_dtype, const float* x_in, const void* vel,
+                const int32_t* src_rows, const int32_t* traj_id, float* x_out, float* logp_out,
+                uint64_t seed, int32_t step, double c_x, double c_v, double noise_std,
+                int logp_mean, RowScratch scratch, cudaStream_t stream);
+
+int launch_score(int n_rows, int elems, int vel_dtype, const float* x, const void* vel,
+                 double p_x, double p_v, float* scores_out, float* preview_out,
+                 RowScratch scratch, cudaStream_t stream);
+
+int launch_ovf(int n_groups, int n, int k, const float* scores, int32_t* keep_idx,
+               int32_t* src_rows, float* sel_var, float* kept_scores, float* adv, float adv_eps,
+               const int32_t* traj_in, int32_t* traj_out, int32_t* status, cudaStream_t stream);
+
+int launch_advantages(int n_groups, int K, const float* rewards, float eps, float* adv,
+                      float* mean, float* std_out, cudaStream_t stream);
+
+int launch_compact(int n_groups, int n_prev, int k, const int32_t* keep_idx, const void* src,
+                   void* dst, size_t row_bytes, cudaStream_t stream);
+
+int launch_iota(int32_t* dst, int n, int32_t base, cudaStream_t stream);
+
+int launch_philox_raw(int64_t n, const uint32_t* ctr, const uint32_t* key, uint32_t* out,
+                      cudaStream_t stream);
+
+int launch_normal_rows(uint64_t seed, int32_t step, int32_t stream_id, int n_rows, int d,
+                       const int32_t* traj_id, float* out, cudaStream_t stream);
+
+}  // namespace pg

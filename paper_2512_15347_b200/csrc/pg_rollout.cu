@@ -1,0 +1,422 @@
+// C ABI of the rollout library: handle, schedule cursor, argument checks, and the host-buffer
+// end-to-end driver.  All arithmetic is in the kernels of pg_step.cu / pg_score.cu / pg_ovf.cu /
+// pg_compact.cu; this file only validates, keeps the cursor and enqueues.
+#include "pg_common.cuh"
+
+#include <atomic>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+namespace pg {
+
+static std::atomic<uint64_t> g_launches{0};
+static thread_local int g_last_cuda_error = 0;
+
+void note_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
+int cuda_fail(cudaError_t e) {
+  g_last_cuda_error = (int)e;
+  (void)cudaGetLastError();   // clear the sticky-less error so later calls start clean
+  return PG_ECUDA;
+}
+
+}  // namespace pg
+
+struct pg_rollout {
+  pg_config cfg;
+  std::vector<int32_t> stage_step, stage_keep;
+  int stage_cur = 0;      // stages already pruned
+  int next_step = 0;
+  int k_cur = 0;          // active trajectories per group
+  int k_prev = 0;         // group size before the most recent prune (for pg_compact)
+  int device = 0;
+  int32_t* d_traj[2] = {nullptr, nullptr};
+  int traj_cur = 0;
+  float* d_partials = nullptr;
+  unsigned int* d_tickets = nullptr;
+  int32_t* d_status = nullptr;
+};
+
+using pg::cuda_fail;
+
+static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+static int validate_config(const pg_config* c) {
+  if (!c) return PG_EINVAL;
+  if (c->n_groups < 1 || c->n_expand < 1 || c->n_expand > PG_MAX_GROUP) return PG_EINVAL;
+  if (c->elems < 4 || (c->elems & 3)) return PG_EINVAL;
+  if (c->n_steps < 1 || c->n_stages < 0) return PG_EINVAL;
+  if (c->n_stages > 0 && (!c->stage_step || !c->stage_keep)) return PG_EINVAL;
+  if (c->vel_dtype != PG_VEL_F32 && c->vel_dtype != PG_VEL_BF16) return PG_EINVAL;
+  if (!(c->adv_eps >= 0.f)) return PG_EINVAL;
+  if (c->group_offset < 0) return PG_EINVAL;
+  const long long ids = ((long long)c->group_offset + c->n_groups) * c->n_expand;
+  if (ids > 0x7FFFFFFFLL) return PG_EINVAL;
+  int prev_step = -1, prev_keep = c->n_expand;
+  for (int i = 0; i < c->n_stages; ++i) {
+    if (c->stage_step[i] <= prev_step || c->stage_step[i] >= c->n_steps) return PG_EINVAL;
+    if (c->stage_keep[i] < 1 || c->stage_keep[i] > prev_keep) return PG_EINVAL;
+    prev_step = c->stage_step[i];
+    prev_keep = c->stage_keep[i];
+  }
+  return PG_OK;
+}
+
+extern "C" {
+
+int pg_rollout_init(const pg_config* cfg, pg_rollout** out) {
+  if (!out) return PG_EINVAL;
+  *out = nullptr;
+  const int rc = validate_config(cfg);
+  if (rc != PG_OK) return rc;
+  pg_rollout* h = new (std::nothrow) pg_rollout();
+  if (!h) return PG_ENOMEM;
+  h->cfg = *cfg;
+  h->stage_step.assign(cfg->stage_step, cfg->stage_step + cfg->n_stages);
+  h->stage_keep.assign(cfg->stage_keep, cfg->stage_keep + cfg->n_stages);
+  h->cfg.stage_step = h->stage_step.data();
+  h->cfg.stage_keep = h->stage_keep.data();
+  h->k_cur = cfg->n_expand;
+  const size_t rows = (size_t)cfg->n_groups * cfg->n_expand;
+  const size_t chunks = (size_t)pg::chunks_per_row(cfg->elems);
+  cudaError_t e = cudaGetDevice(&h->device);
+  if (e == cudaSuccess) e = cudaMalloc(&h->d_traj[0], rows * sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&h->d_traj[1], rows * sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&h->d_partials, rows * chunks * sizeof(float));
+  if (e == cudaSuccess) e = cudaMalloc(&h->d_tickets, rows * sizeof(unsigned int));
+  if (e == cudaSuccess) e = cudaMalloc(&h->d_status, sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMemset(h->d_tickets, 0, rows * sizeof(unsigned int));
+  if (e == cudaSuccess) e = cudaMemset(h->d_status, 0, sizeof(int32_t));
+  int lrc = PG_OK;
+  if (e == cudaSuccess)
+    lrc = pg::launch_iota(h->d_traj[0], (int)rows, cfg->group_offset * cfg->n_expand, nullptr);
+  if (e == cudaSuccess && lrc == PG_OK) e = cudaStreamSynchronize(nullptr);
+  if (e != cudaSuccess || lrc != PG_OK) {
+    const int code = (e == cudaErrorMemoryAllocation) ? PG_ENOMEM : (e != cudaSuccess ? cuda_fail(e) : lrc);
+    pg_rollout_destroy(h);
+    return code;
+  }
+  *out = h;
+  return PG_OK;
+}
+
+int pg_rollout_destroy(pg_rollout* h) {
+  if (!h) return PG_OK;
+  cudaFree(h->d_traj[0]);
+  cudaFree(h->d_traj[1]);
+  cudaFree(h->d_partials);
+  cudaFree(h->d_tickets);
+  cudaFree(h->d_status);
+  delete h;
+  return PG_OK;
+}
+
+int pg_rollout_reset(pg_rollout* h, void* stream) {
+  if (!h) return PG_EINVAL;
+  cudaStream_t st = (cudaStream_t)stream;
+  const int rows = h->cfg.n_groups * h->cfg.n_expand;
+  h->stage_cur = 0;
+  h->next_step = 0;
+  h->k_cur = h->cfg.n_expand;
+  h->k_prev = 0;
+  h->traj_cur = 0;
+  PG_CUDA(cudaMemsetAsync(h->d_status, 0, sizeof(int32_t), st));
+  PG_CUDA(cudaMemsetAsync(h->d_tickets, 0, (size_t)rows * sizeof(unsigned int), st));
+  return pg::launch_iota(h->d_traj[0], rows, h->cfg.group_offset * h->cfg.n_expand, st);
+}
+
+int pg_rollout_status(pg_rollout* h, int32_t* n_active, int32_t* next_step, int32_t* device_status) {
+  if (!h) return PG_EINVAL;
+  PG_CUDA(cudaDeviceSynchronize());
+  int32_t st = 0;
+  PG_CUDA(cudaMemcpy(&st, h->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost));
+  if (n_active) *n_active = h->cfg.n_groups * h->k_cur;
+  if (next_step) *next_step = h->next_step;
+  if (device_status) *device_status = st;
+  if (st & 2) return PG_ETIMEOUT;
+  if (st & 1) return PG_ENONFINITE;
+  return PG_OK;
+}
+
+int pg_step(pg_rollout* h, int32_t step, const pg_step_coef* coef, const float* x_in,
+            const void* vel, const int32_t* src_rows, float* x_out, float* logp_out, void* stream) {
+  if (!h || !coef || !x_in || !vel || !x_out || !logp_out) return PG_EINVAL;
+  if (!aligned16(x_in) || !aligned16(vel) || !aligned16(x_out)) return PG_EINVAL;
+  if (src_rows && x_in == x_out) return PG_EINVAL;
+  if (!(coef->noise_std >= 0.0) || !std::isfinite(coef->c_x) || !std::isfinite(coef->c_v) ||
+      !std::isfinite(coef->noise_std))
+    return PG_EINVAL;
+  if (step != h->next_step || step >= h->cfg.n_steps) return PG_ESTATE;
+  if (h->stage_cur < h->cfg.n_stages && h->stage_step[h->stage_cur] == step) return PG_ESTATE;
+  const int rows = h->cfg.n_groups * h->k_cur;
+  pg::RowScratch scratch{h->d_partials, h->d_tickets};
+  const int rc = pg::launch_step(rows, h->cfg.elems, h->cfg.vel_dtype, x_in, vel, src_rows,
+                                 h->d_traj[h->traj_cur], x_out, logp_out, h->cfg.seed, step,
+                                 coef->c_x, coef->c_v, coef->noise_std, h->cfg.logp_mean, scratch,
+                                 (cudaStream_t)stream);
+  if (rc == PG_OK) h->next_step = step + 1;
+  return rc;
+}
+
+int pg_score(pg_rollout* h, const pg_preview_coef* coef, const float* x, const void* vel,
+             float* scores_out, float* preview_out, void* stream) {
+  if (!h || !coef || !x || !scores_out) return PG_EINVAL;
+  if (!std::isfinite(coef->p_x) || !std::isfinite(coef->p_v)) return PG_EINVAL;
+  if (coef->p_v != 0.0 && !vel) return PG_EINVAL;
+  if (!aligned16(x) || !aligned16(vel) || !aligned16(preview_out)) return PG_EINVAL;
+  const int rows = h->cfg.n_groups * h->k_cur;
+  pg::RowScratch scratch{h->d_partials, h->d_tickets};
+  return pg::launch_score(rows, h->cfg.elems, h->cfg.vel_dtype, x, vel, coef->p_x, coef->p_v,
+                          scores_out, preview_out, scratch, (cudaStream_t)stream);
+}
+
+int pg_prune_ovf(pg_rollout* h, int32_t stage, const float* scores, int32_t* keep_idx,
+                 int32_t* src_rows, float* sel_var, void* stream) {
+  if (!h || !scores || !keep_idx) return PG_EINVAL;
+  if (stage != h->stage_cur || stage >= h->cfg.n_stages) return PG_ESTATE;
+  if (h->stage_step[stage] != h->next_step) return PG_ESTATE;
+  const int n = h->k_cur, k = h->stage_keep[stage];
+  const int rc = pg::launch_ovf(h->cfg.n_groups, n, k, scores, keep_idx, src_rows, sel_var, nullptr,
+                                nullptr, 0.f, h->d_traj[h->traj_cur], h->d_traj[h->traj_cur ^ 1],
+                                h->d_status, (cudaStream_t)stream);
+  if (rc != PG_OK) return rc;
+  h->traj_cur ^= 1;
+  h->k_prev = n;
+  h->k_cur = k;
+  h->stage_cur = stage + 1;
+  return PG_OK;
+}
+
+int pg_compact(pg_rollout* h, const int32_t* keep_idx, const void* src, void* dst, size_t row_bytes,
+               void* stream) {
+  if (!h || !keep_idx || !src || !dst || row_bytes == 0) return PG_EINVAL;
+  if (h->k_prev == 0) return PG_ESTATE;
+  const size_t src_bytes = (size_t)h->cfg.n_groups * h->k_prev * row_bytes;
+  const size_t dst_bytes = (size_t)h->cfg.n_groups * h->k_cur * row_bytes;
+  const uintptr_t s = (uintptr_t)src, d = (uintptr_t)dst;
+  if (s < d + dst_bytes && d < s + src_bytes) return PG_EINVAL;   // overlap
+  return pg::launch_compact(h->cfg.n_groups, h->k_prev, h->k_cur, keep_idx, src, dst, row_bytes,
+                            (cudaStream_t)stream);
+}
+
+int pg_advantages(pg_rollout* h, const float* rewards, float* adv, float* mean, float* std,
+                  void* stream) {
+  if (!h || !rewards || !adv) return PG_EINVAL;
+  return pg::launch_advantages(h->cfg.n_groups, h->k_cur, rewards, h->cfg.adv_eps, adv, mean, std,
+                               (cudaStream_t)stream);
+}
+
+int pg_ovf_select_batched(int32_t n_groups, int32_t n, int32_t k, const float* scores,
+                          int32_t* keep_idx, float* kept_scores, float* adv, float adv_eps,
+                          int32_t* status, void* stream) {
+  if (n_groups < 0 || n < 1 || n > PG_MAX_GROUP || k < 1 || k > n) return PG_EINVAL;
+  if (!scores || !keep_idx || !(adv_eps >= 0.f)) return PG_EINVAL;
+  return pg::launch_ovf(n_groups, n, k, scores, keep_idx, nullptr, nullptr, kept_scores, adv,
+                        adv_eps, nullptr, nullptr, status, (cudaStream_t)stream);
+}
+
+int pg_rollout_traj_ids(pg_rollout* h, int32_t* dst, void* stream) {
+  if (!h || !dst) return PG_EINVAL;
+  PG_CUDA(cudaMemcpyAsync(dst, h->d_traj[h->traj_cur],
+                          (size_t)h->cfg.n_groups * h->k_cur * sizeof(int32_t),
+                          cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
+  return PG_OK;
+}
+
+int pg_philox_raw(int64_t n, const uint32_t* ctr, const uint32_t* key, uint32_t* out, void* stream) {
+  if (n < 0 || (n > 0 && (!ctr || !key || !out)) || !aligned16(out)) return PG_EINVAL;
+  return pg::launch_philox_raw(n, ctr, key, out, (cudaStream_t)stream);
+}
+
+int pg_normal_rows(uint64_t seed, int32_t step, int32_t stream_id, int32_t n_rows, int32_t d,
+                   const int32_t* traj_id, float* out, void* stream) {
+  if (n_rows < 0 || d < 4 || (d & 3) || step < 0 || stream_id < 0) return PG_EINVAL;
+  if (n_rows > 0 && (!traj_id || !out || !aligned16(out))) return PG_EINVAL;
+  return pg::launch_normal_rows(seed, step, stream_id, n_rows, d, traj_id, out, (cudaStream_t)stream);
+}
+
+const char* pg_strerror(int code) {
+  switch (code) {
+    case PG_OK: return "ok";
+    case PG_EINVAL: return "invalid argument (null pointer, shape, alignment or overlap)";
+    case PG_ESTATE: return "call out of sequence for the rollout schedule";
+    case PG_ECUDA: return "CUDA runtime error (see pg_last_cuda_error)";
+    case PG_ENONFINITE: return "non-finite scores were seen by the selection";
+    case PG_ETIMEOUT: return "a bounded device-side wait expired";
+    case PG_ENOMEM: return "out of memory";
+    default: return "unknown error code";
+  }
+}
+
+int pg_last_cuda_error(void) { return pg::g_last_cuda_error; }
+uint64_t pg_launch_count(void) { return pg::g_launches.load(std::memory_order_relaxed); }
+
+// ---------------------------------------------------------------- host-buffer driver
+
+static size_t round256(size_t b) { return (b + 255) & ~(size_t)255; }
+
+struct HostPlan {
+  size_t rows0, vel_elem, x_bytes, v_bytes, total_logp, total_keep;
+  size_t off_x[2], off_v[2], off_scores, off_keep, off_src, off_logp, off_rewards, off_adv,
+      off_traj, total;
+};
+
+static HostPlan make_plan(const pg_config* c) {
+  HostPlan p;
+  p.rows0 = (size_t)c->n_groups * c->n_expand;
+  p.vel_elem = c->vel_dtype == PG_VEL_BF16 ? 2 : 4;
+  p.x_bytes = p.rows0 * c->elems * sizeof(float);
+  p.v_bytes = p.rows0 * c->elems * p.vel_elem;
+  p.total_logp = 0;
+  p.total_keep = 0;
+  int k = c->n_expand, si = 0;
+  for (int s = 0; s < c->n_steps; ++s) {
+    if (si < c->n_stages && c->stage_step[si] == s) {
+      k = c->stage_keep[si++];
+      p.total_keep += (size_t)c->n_groups * k;
+    }
+    p.total_logp += (size_t)c->n_groups * k;
+  }
+  size_t o = 0;
+  for (int i = 0; i < 2; ++i) { p.off_x[i] = o; o += round256(p.x_bytes); }
+  for (int i = 0; i < 2; ++i) { p.off_v[i] = o; o += round256(p.v_bytes); }
+  p.off_scores = o;  o += round256(p.rows0 * 4);
+  p.off_keep = o;    o += round256((p.total_keep + 1) * 4);
+  p.off_src = o;     o += round256(p.rows0 * 4);
+  p.off_logp = o;    o += round256(p.total_logp * 4);
+  p.off_rewards = o; o += round256(p.rows0 * 4);
+  p.off_adv = o;     o += round256(p.rows0 * 4);
+  p.off_traj = o;    o += round256(p.rows0 * 4);
+  p.total = o;
+  return p;
+}
+
+size_t pg_rollout_host_workspace_bytes(const pg_config* cfg) {
+  if (validate_config(cfg) != PG_OK) return 0;
+  return make_plan(cfg).total;
+}
+
+int pg_rollout_host(const pg_config* cfg, const pg_step_coef* step_coef,
+                    const pg_preview_coef* preview_coef, const float* x0,
+                    const void* const* vel_steps, const float* const* stage_scores,
+                    const float* final_rewards, float* x_final, float* logp, int32_t* keep_idx,
+                    float* adv, int32_t* traj_id, void* workspace, size_t workspace_bytes) {
+  int rc = validate_config(cfg);
+  if (rc != PG_OK) return rc;
+  if (!step_coef || !x0 || !vel_steps || !workspace || !aligned16(workspace)) return PG_EINVAL;
+  if (cfg->n_stages > 0 && !preview_coef && !stage_scores) return PG_EINVAL;
+  const HostPlan pl = make_plan(cfg);
+  if (workspace_bytes < pl.total) return PG_EINVAL;
+  for (int s = 0; s < cfg->n_steps; ++s)
+    if (!vel_steps[s]) return PG_EINVAL;
+
+  unsigned char* ws = (unsigned char*)workspace;
+  float* d_x[2] = {(float*)(ws + pl.off_x[0]), (float*)(ws + pl.off_x[1])};
+  void* d_v[2] = {ws + pl.off_v[0], ws + pl.off_v[1]};
+  float* d_scores = (float*)(ws + pl.off_scores);
+  int32_t* d_keep = (int32_t*)(ws + pl.off_keep);
+  int32_t* d_src = (int32_t*)(ws + pl.off_src);
+  float* d_logp = (float*)(ws + pl.off_logp);
+  float* d_rewards = (float*)(ws + pl.off_rewards);
+  float* d_adv = (float*)(ws + pl.off_adv);
+  int32_t* d_traj = (int32_t*)(ws + pl.off_traj);
+
+  pg_rollout* h = nullptr;
+  rc = pg_rollout_init(cfg, &h);
+  if (rc != PG_OK) return rc;
+  cudaStream_t compute = nullptr, copy = nullptr;
+  cudaEvent_t v_ready[2] = {nullptr, nullptr}, v_free[2] = {nullptr, nullptr};
+  auto cleanup = [&](int code) {
+    cudaDeviceSynchronize();
+    for (int i = 0; i < 2; ++i) {
+      if (v_ready[i]) cudaEventDestroy(v_ready[i]);
+      if (v_free[i]) cudaEventDestroy(v_free[i]);
+    }
+    if (compute) cudaStreamDestroy(compute);
+    if (copy) cudaStreamDestroy(copy);
+    pg_rollout_destroy(h);
+    return code;
+  };
+#define PG_TRY_CUDA(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return cleanup(cuda_fail(e_)); } while (0)
+#define PG_TRY(call) do { int r_ = (call); if (r_ != PG_OK) return cleanup(r_); } while (0)
+  PG_TRY_CUDA(cudaStreamCreateWithFlags(&compute, cudaStreamNonBlocking));
+  PG_TRY_CUDA(cudaStreamCreateWithFlags(&copy, cudaStreamNonBlocking));
+  for (int i = 0; i < 2; ++i) {
+    PG_TRY_CUDA(cudaEventCreateWithFlags(&v_ready[i], cudaEventDisableTiming));
+    PG_TRY_CUDA(cudaEventCreateWithFlags(&v_free[i], cudaEventDisableTiming));
+  }
+
+  // rows alive when the prediction of step s is made
+  std::vector<int> rows_pred(cfg->n_steps);
+  {
+    int k = cfg->n_expand, si = 0;
+    for (int s = 0; s < cfg->n_steps; ++s) {
+      rows_pred[s] = cfg->n_groups * k;
+      if (si < cfg->n_stages && cfg->stage_step[si] == s) k = cfg->stage_keep[si++];
+    }
+  }
+  auto prefetch = [&](int s) -> cudaError_t {
+    const int b = s & 1;
+    cudaError_t e = cudaSuccess;
+    if (s >= 2) e = cudaStreamWaitEvent(copy, v_free[b], 0);
+    if (e == cudaSuccess)
+      e = cudaMemcpyAsync(d_v[b], vel_steps[s], (size_t)rows_pred[s] * cfg->elems * pl.vel_elem,
+                          cudaMemcpyHostToDevice, copy);
+    if (e == cudaSuccess) e = cudaEventRecord(v_ready[b], copy);
+    return e;
+  };
+
+  PG_TRY_CUDA(cudaMemcpyAsync(d_x[0], x0, pl.x_bytes, cudaMemcpyHostToDevice, compute));
+  PG_TRY_CUDA(prefetch(0));
+  int cur = 0, stage = 0;
+  size_t logp_off = 0, keep_off = 0;
+  for (int s = 0; s < cfg->n_steps; ++s) {
+    if (s + 1 < cfg->n_steps) PG_TRY_CUDA(prefetch(s + 1));
+    const int b = s & 1;
+    PG_TRY_CUDA(cudaStreamWaitEvent(compute, v_ready[b], 0));
+    const int32_t* src = nullptr;
+    if (stage < cfg->n_stages && cfg->stage_step[stage] == s) {
+      const int rows = cfg->n_groups * h->k_cur;
+      if (stage_scores && stage_scores[stage]) {
+        PG_TRY_CUDA(cudaMemcpyAsync(d_scores, stage_scores[stage], (size_t)rows * 4,
+                                    cudaMemcpyHostToDevice, compute));
+      } else {
+        if (!preview_coef) return cleanup(PG_EINVAL);
+        PG_TRY(pg_score(h, &preview_coef[stage], d_x[cur], d_v[b], d_scores, nullptr, compute));
+      }
+      PG_TRY(pg_prune_ovf(h, stage, d_scores, d_keep + keep_off, d_src, nullptr, compute));
+      keep_off += (size_t)cfg->n_groups * h->k_cur;
+      src = d_src;
+      ++stage;
+    }
+    float* x_out = src ? d_x[cur ^ 1] : d_x[cur];
+    PG_TRY(pg_step(h, s, &step_coef[s], d_x[cur], d_v[b], src, x_out, d_logp + logp_off, compute));
+    if (src) cur ^= 1;
+    logp_off += (size_t)cfg->n_groups * h->k_cur;
+    PG_TRY_CUDA(cudaEventRecord(v_free[b], compute));
+  }
+  const size_t rows_final = (size_t)cfg->n_groups * h->k_cur;
+  if (final_rewards) {
+    PG_TRY_CUDA(cudaMemcpyAsync(d_rewards, final_rewards, rows_final * 4, cudaMemcpyHostToDevice, compute));
+  } else {
+    const pg_preview_coef id = {1.0, 0.0};
+    PG_TRY(pg_score(h, &id, d_x[cur], nullptr, d_rewards, nullptr, compute));
+  }
+  PG_TRY(pg_advantages(h, d_rewards, d_adv, nullptr, nullptr, compute));
+  PG_TRY(pg_rollout_traj_ids(h, d_traj, compute));
+  if (x_final) PG_TRY_CUDA(cudaMemcpyAsync(x_final, d_x[cur], rows_final * cfg->elems * 4, cudaMemcpyDeviceToHost, compute));
+  if (logp) PG_TRY_CUDA(cudaMemcpyAsync(logp, d_logp, pl.total_logp * 4, cudaMemcpyDeviceToHost, compute));
+  if (keep_idx && pl.total_keep) PG_TRY_CUDA(cudaMemcpyAsync(keep_idx, d_keep, pl.total_keep * 4, cudaMemcpyDeviceToHost, compute));
+  if (adv) PG_TRY_CUDA(cudaMemcpyAsync(adv, d_adv, rows_final * 4, cudaMemcpyDeviceToHost, compute));
+  if (traj_id) PG_TRY_CUDA(cudaMemcpyAsync(traj_id, d_traj, rows_final * 4, cudaMemcpyDeviceToHost, compute));
+  PG_TRY_CUDA(cudaStreamSynchronize(compute));
+  int32_t st = 0;
+  PG_TRY_CUDA(cudaMemcpy(&st, h->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost));
+  return cleanup((st & 2) ? PG_ETIMEOUT : (st & 1) ? PG_ENONFINITE : PG_OK);
+#undef PG_TRY
+#undef PG_TRY_CUDA
+}
+
+}  // extern "C"

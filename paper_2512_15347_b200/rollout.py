@@ -1,0 +1,146 @@
+"""Thin driver over the C ABI: owns the device buffers of one rollout batch and issues the
+library calls in schedule order.  Allocation and streams are torch's; every number is computed
+by the library's kernels.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+from typing import Callable, List, Optional, Sequence, Tuple
+
+import torch
+
+from . import binding as B
+
+
+@dataclass
+class RolloutOutput:
+    x_final: torch.Tensor                 # [G*K, d] fp32
+    logp: List[torch.Tensor]              # per step [rows taking that step] fp32
+    traj_id: torch.Tensor                 # [G*K] int32
+    stage_scores: List[torch.Tensor] = field(default_factory=list)
+    stage_keep: List[torch.Tensor] = field(default_factory=list)
+    stage_var: List[torch.Tensor] = field(default_factory=list)
+    rewards: Optional[torch.Tensor] = None
+    adv: Optional[torch.Tensor] = None
+    mean: Optional[torch.Tensor] = None
+    std: Optional[torch.Tensor] = None
+
+
+class Rollout:
+    """One Expand-and-Prune batch on the current CUDA device."""
+
+    def __init__(self, n_groups: int, n_expand: int, elems: int, n_steps: int,
+                 stages: Sequence[Tuple[int, int]], seed: int, vel_dtype: torch.dtype,
+                 adv_eps: float = 1e-6, group_offset: int = 0, logp_mean: bool = False):
+        if not torch.cuda.is_available():
+            raise RuntimeError("the rollout library needs a CUDA device; there is no CPU path")
+        self.G, self.N0, self.d, self.T = n_groups, n_expand, elems, n_steps
+        self.stages = [(int(s), int(k)) for s, k in stages]
+        self.vel_dtype = vel_dtype
+        vd = B.VEL_BF16 if vel_dtype == torch.bfloat16 else B.VEL_F32
+        self.cfg = B.make_config(n_groups, n_expand, elems, n_steps, self.stages, seed, vd,
+                                 group_offset=group_offset, logp_mean=logp_mean, adv_eps=adv_eps)
+        self.h = B.rollout_init(self.cfg)
+        dev = torch.device("cuda", torch.cuda.current_device())
+        rows = n_groups * n_expand
+        self.dev = dev
+        self.x = [torch.empty(rows, elems, device=dev, dtype=torch.float32) for _ in range(2)]
+        self.cur = 0
+        self.k_cur = n_expand
+        self.scores = torch.empty(rows, device=dev, dtype=torch.float32)
+        self.src_rows = torch.empty(rows, device=dev, dtype=torch.int32)
+        self.rewards = torch.empty(rows, device=dev, dtype=torch.float32)
+        total = 0
+        k = n_expand
+        st = dict(self.stages)
+        self.rows_at = []
+        for s in range(n_steps):
+            k = st.get(s, k)
+            self.rows_at.append(n_groups * k)
+            total += n_groups * k
+        self.logp_all = torch.empty(total, device=dev, dtype=torch.float32)
+        self.keep = [torch.empty(n_groups * k, device=dev, dtype=torch.int32) for _, k in self.stages]
+        self.sel_var = [torch.empty(n_groups, device=dev, dtype=torch.float32) for _ in self.stages]
+        self.adv = torch.empty(n_groups * (self.stages[-1][1] if self.stages else n_expand),
+                               device=dev, dtype=torch.float32)
+        self.mean = torch.empty(n_groups, device=dev, dtype=torch.float32)
+        self.std = torch.empty(n_groups, device=dev, dtype=torch.float32)
+
+    def close(self):
+        if getattr(self, "h", None):
+            torch.cuda.synchronize()
+            B.rollout_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def n_active(self) -> int:
+        return self.G * self.k_cur
+
+    def x_active(self) -> torch.Tensor:
+        return self.x[self.cur][: self.n_active]
+
+    def reset(self, x0: torch.Tensor):
+        B.rollout_reset(self.h)
+        self.cur = 0
+        self.k_cur = self.N0
+        self.x[0].copy_(x0)
+
+    def run(self, x0: torch.Tensor,
+            step_coef: Callable[[int], Tuple[float, float, float]],
+            preview_coef: Callable[[int], Tuple[float, float]],
+            velocity: Callable[[int, torch.Tensor], torch.Tensor],
+            external_scores: Optional[Callable[[int], torch.Tensor]] = None,
+            final_rewards: Optional[Callable[[], torch.Tensor]] = None,
+            record_scores: bool = False) -> RolloutOutput:
+        """Runs the whole schedule.  ``velocity(step, x_active)`` returns the prediction for the
+        currently active rows; ``external_scores(stage)`` / ``final_rewards()`` return device
+        fp32 tensors when the scores come from outside (else the preview mean / latent mean)."""
+        self.reset(x0)
+        out = RolloutOutput(x_final=None, logp=[], traj_id=None)
+        stage_i, off = 0, 0
+        for s in range(self.T):
+            vel = velocity(s, self.x_active())
+            src = None
+            if stage_i < len(self.stages) and self.stages[stage_i][0] == s:
+                if external_scores is not None:
+                    sc = external_scores(stage_i)
+                else:
+                    sc = self.scores[: self.n_active]
+                    B.score(self.h, preview_coef(s), self.x[self.cur], vel, sc)
+                if record_scores:
+                    out.stage_scores.append(sc.clone())
+                B.prune_ovf(self.h, stage_i, sc, self.keep[stage_i], self.src_rows,
+                            self.sel_var[stage_i])
+                self.k_cur = self.stages[stage_i][1]
+                src = self.src_rows
+                stage_i += 1
+            rows = self.n_active
+            lp = self.logp_all[off: off + rows]
+            if src is not None:
+                B.step(self.h, s, step_coef(s), self.x[self.cur], vel, src, self.x[self.cur ^ 1], lp)
+                self.cur ^= 1
+            else:
+                B.step(self.h, s, step_coef(s), self.x[self.cur], vel, None, self.x[self.cur], lp)
+            out.logp.append(lp)
+            off += rows
+        rows = self.n_active
+        if final_rewards is not None:
+            rw = final_rewards()
+        else:
+            rw = self.rewards[:rows]
+            B.score(self.h, (1.0, 0.0), self.x[self.cur], None, rw)
+        B.advantages(self.h, rw, self.adv, self.mean, self.std)
+        ids = torch.empty(rows, device=self.dev, dtype=torch.int32)
+        B.rollout_traj_ids(self.h, ids)
+        out.x_final = self.x_active()
+        out.traj_id = ids
+        out.stage_keep = list(self.keep)
+        out.stage_var = list(self.sel_var)
+        out.rewards, out.adv, out.mean, out.std = rw, self.adv, self.mean, self.std
+        return out

@@ -1,0 +1,132 @@
+"""Shared helpers of the GPU parity tests: error metrics and oracle/GPU drivers."""
+import numpy as np
+import torch
+
+import oracle
+from paper_2512_15347_b200 import workloads as wl
+
+# Tolerances (fp32 arithmetic on the device against the fp64 oracle, identical input bits):
+#   latents   max_e |a-b| / max(|b_e|, rms(b_row))  <= 1e-5
+#   log-probs |a-b| / max(|b|, 1e-30)               <= 1e-5
+#   scores    |a-b| <= 1e-6 (selection may differ only where score gaps are below 1e-6)
+LATENT_TOL = 1e-5
+LOGP_TOL = 1e-5
+SCORE_GAP = 1e-6
+
+
+def latent_err(a: np.ndarray, b: np.ndarray) -> float:
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    if a.size == 0:
+        return 0.0
+    rms = np.sqrt((b * b).mean(axis=1, keepdims=True))
+    den = np.maximum(np.abs(b), np.maximum(rms, 1e-30))
+    return float((np.abs(a - b) / den).max())
+
+
+def rel_err(a, b) -> float:
+    a = np.asarray(a, dtype=np.float64)
+    b = np.asarray(b, dtype=np.float64)
+    if a.size == 0:
+        return 0.0
+    return float((np.abs(a - b) / np.maximum(np.abs(b), 1e-30)).max())
+
+
+def to_dev(a: np.ndarray) -> torch.Tensor:
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def vel_to_dev(v: np.ndarray) -> torch.Tensor:
+    if v.dtype == np.uint16:
+        return torch.from_numpy(v.view(np.int16)).cuda().view(torch.bfloat16)
+    return torch.from_numpy(v).cuda()
+
+
+class SharedInputs:
+    """Generates every input once on the CPU and serves the same bytes to both sides."""
+
+    def __init__(self, w: wl.Workload):
+        self.w = w
+        self.x0 = wl.initial_latents(w).numpy()
+        self.affine = wl.affine_field(w) if w.velocity == "affine" else None
+        self._vel = {}
+
+    def vel_numpy(self, step: int, x: np.ndarray) -> np.ndarray:
+        w = self.w
+        if w.velocity == "affine":
+            a, b = self.affine
+            return wl.affine_velocity(torch.from_numpy(x), a, b).numpy()
+        if step not in self._vel:
+            rows = w.n_groups * w.rows_before(step)
+            self._vel[step] = wl.as_numpy_velocity(wl.normal_velocity(w, step, rows))
+        v = self._vel[step]
+        assert v.shape[0] == x.shape[0]
+        return v
+
+    def vel_device(self, step: int, x: torch.Tensor) -> torch.Tensor:
+        w = self.w
+        if w.velocity == "affine":
+            a, b = self.affine
+            return wl.affine_velocity(x, a.cuda(), b.cuda())
+        return vel_to_dev(self.vel_numpy(step, np.empty((x.shape[0], 0))))
+
+
+def run_oracle(w: wl.Workload, inp: SharedInputs, keep_steps=False):
+    ext = None
+    fin = None
+    if w.scores == "external":
+        ext = lambda stage, traj: wl.sd3_stage_scores(w, stage, traj)
+        fin = lambda x, traj: wl.sd3_stage_scores(w, 99, traj)
+    return oracle.rollout(inp.x0, w.n_groups, w.n_expand, w.n_steps, w.stages, w.seed,
+                          w.step_coef, w.preview_coef,
+                          lambda s, x, traj: inp.vel_numpy(s, x),
+                          external_scores=ext, final_rewards=fin, adv_eps=w.adv_eps,
+                          keep_steps=keep_steps)
+
+
+def run_gpu(w: wl.Workload, inp: SharedInputs, record_scores=True):
+    from paper_2512_15347_b200.rollout import Rollout
+    dt = torch.bfloat16 if w.vel_dtype == "bf16" else torch.float32
+    ro = Rollout(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, dt, adv_eps=w.adv_eps)
+    ext = None
+    fin = None
+    if w.scores == "external":
+        from paper_2512_15347_b200 import binding as B
+
+        def ext(stage):
+            ids = torch.empty(ro.n_active, device="cuda", dtype=torch.int32)
+            B.rollout_traj_ids(ro.h, ids)
+            return to_dev(wl.sd3_stage_scores(w, stage, ids.cpu().numpy()))
+
+        def fin():
+            ids = torch.empty(ro.n_active, device="cuda", dtype=torch.int32)
+            B.rollout_traj_ids(ro.h, ids)
+            return to_dev(wl.sd3_stage_scores(w, 99, ids.cpu().numpy()))
+    out = ro.run(to_dev(inp.x0), w.step_coef, w.preview_coef,
+                 lambda s, x: inp.vel_device(s, x), external_scores=ext, final_rewards=fin,
+                 record_scores=record_scores)
+    torch.cuda.synchronize()
+    return ro, out
+
+
+def compare_rollouts(w: wl.Workload, ref, out):
+    """Element-by-element comparison of a GPU rollout with the oracle's."""
+    for i, (s, k) in enumerate(w.stages):
+        got_keep = out.stage_keep[i].cpu().numpy().reshape(w.n_groups, k)
+        if out.stage_scores:
+            got_sc = out.stage_scores[i].cpu().numpy().reshape(ref.stage_scores[i].shape)
+            assert np.abs(got_sc.astype(np.float64) - ref.stage_scores[i].astype(np.float64)).max() <= SCORE_GAP
+            # given the device's own scores the selection must be the oracle's, bit for bit
+            keep_again, _ = oracle.ovf_select(got_sc, k)
+            np.testing.assert_array_equal(got_keep, keep_again)
+        np.testing.assert_array_equal(got_keep, ref.stage_keep[i])
+    np.testing.assert_array_equal(out.traj_id.cpu().numpy(), ref.traj_id)
+    worst_lp = 0.0
+    for s in range(w.n_steps):
+        worst_lp = max(worst_lp, rel_err(out.logp[s].cpu().numpy(), ref.logp[s]))
+    assert worst_lp <= LOGP_TOL, worst_lp
+    e = latent_err(out.x_final.cpu().numpy(), ref.x_final)
+    assert e <= LATENT_TOL, e
+    k = w.final_keep
+    np.testing.assert_allclose(out.adv.cpu().numpy().reshape(w.n_groups, k), ref.adv, rtol=2e-4, atol=2e-5)
+    return worst_lp, e
