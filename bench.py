@@ -1,0 +1,397 @@
+#!/usr/bin/env python
+"""Benchmark of the Expand-and-Prune rollout hot path.
+
+One "step" of this benchmark is one whole rollout of the large workload (64 prompt groups,
+64 -> 32 -> 16 (-> 16) trajectories pruned at steps 2, 5, 8 of 28, 16x128x128 fp32 latents, bf16
+predictions): SDE step + log-prob at every step, latent scoring + OVF + (folded) compaction at
+every stage, group advantages at the end.  The reported value is latent-steps per second
+(one latent-step = one trajectory advanced by one SDE step, log-prob included).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+With N > 1 (launched by torch.distributed.run, one rank per GPU) every rank runs its own 64
+groups (weak scaling, groups are independent, no data-path collective); times are taken on the
+device and the maximum over ranks is used.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import math
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "latent-steps/s (SDE step+logprob+OVF prune)"
+UNIT = "latent-steps/s"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        try:
+            return float(json.load(open(path))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        rows = [r for r in self.rows if t0 - 0.05 <= r[0] <= t1 + 0.15] or self.rows
+        for _, line in rows:
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown",
+                                  "sw_power_cap"), f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2] if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------ CPU oracle timing
+
+class OracleSample:
+    """A bounded sample of the workload for the CPU oracle: the first `groups` prompt groups with
+    the full schedule and full-length latents (groups are independent, cost is linear in groups)."""
+
+    def __init__(self, w, groups: int):
+        from paper_2512_15347_b200 import workloads as wl
+        self.w = w
+        self.sw = wl.scaled(w, n_groups=groups)
+        self.x0 = wl.initial_latents(self.sw).numpy()
+        self.vels = [wl.as_numpy_velocity(wl.normal_velocity(self.sw, s, groups * w.rows_before(s)))
+                     for s in range(w.n_steps)]
+        self.desc = (f"first {groups} of {w.n_groups} prompt groups, full schedule, full-length latents "
+                     f"({self.sw.traj_steps} of {w.traj_steps} latent-steps)")
+
+    def run(self) -> float:
+        """One oracle rollout of the sample; returns seconds."""
+        import oracle
+        sw = self.sw
+        t0 = time.perf_counter()
+        oracle.rollout(self.x0, sw.n_groups, sw.n_expand, sw.n_steps, sw.stages, sw.seed, sw.step_coef,
+                       sw.preview_coef, lambda s, x, traj: self.vels[s], adv_eps=sw.adv_eps)
+        return time.perf_counter() - t0
+
+
+ORACLE_GROUPS = 8
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    from paper_2512_15347_b200 import workloads as wl
+    w = wl.WORKLOADS[args.workload]
+    sample = OracleSample(w, min(ORACLE_GROUPS, w.n_groups))
+    small = OracleSample(w, 1)
+    for _ in range(max(args.warmup, 0)):
+        small.run()
+    times = [sample.run() for _ in range(args.steps)]
+    mean_sec = sum(times) / len(times)
+    value = sample.sw.traj_steps / mean_sec
+    threads = oracle.num_threads()
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": mean_sec * 1e3,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": _config(w, args),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": sample.desc + "; warm-up on 1 group"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+def _config(w, args):
+    return {"workload": f"{w.name}: {w.n_groups} groups x {w.n_expand} -> "
+                        + " -> ".join(str(k) for _, k in w.stages)
+                        + f" at steps {[s for s, _ in w.stages]} of {w.n_steps}, d={w.elems}, "
+                        f"fp32 latents, {w.vel_dtype} predictions, seed {w.seed}",
+            "groups_per_gpu": w.n_groups, "latent_steps_per_rollout": w.traj_steps,
+            "l2": "inputs larger than L2: no flush (state %.2f GB, predictions %.2f GB per rollout)"
+                  % (w.n_groups * w.n_expand * w.elems * 4 / 1e9,
+                     w.element_steps * (2 if w.vel_dtype == "bf16" else 4) / 1e9),
+            "parallelism": f"groups sharded over {args.gpus} GPU(s), no collective"}
+
+
+# ------------------------------------------------------------------ GPU arm
+
+def run_ours(args):
+    import torch
+    from paper_2512_15347_b200 import binding as B
+    from paper_2512_15347_b200 import workloads as wl
+    from paper_2512_15347_b200.rollout import Rollout
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    w = wl.WORKLOADS[args.workload]
+    if args.groups:
+        w = wl.scaled(w, n_groups=args.groups, name=f"{w.name}[{args.groups} groups]")
+
+    cpu_base = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        # before the first CUDA call: the oracle's OpenMP team is created in a clean process
+        import oracle
+        sample = OracleSample(w, min(ORACLE_GROUPS, w.n_groups))
+        sec = min(sample.run() for _ in range(2))
+        cpu_base = {"value": sample.sw.traj_steps / sec, "unit": UNIT, "cores": oracle.num_threads(),
+                    "kind": "oracle", "sample": sample.desc + f"; best of 2 runs, {sec:.1f} s each"}
+        del sample
+
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    B.lib()
+    dev = torch.device("cuda", local)
+    from dataclasses import replace
+    wr = replace(w, seed=w.seed + 1000 * rank)
+
+    dt = torch.bfloat16 if w.vel_dtype == "bf16" else torch.float32
+    ro = Rollout(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, dt, adv_eps=w.adv_eps,
+                 group_offset=rank * w.n_groups)
+    x0 = wl.initial_latents(wr, device=dev)
+    vels = [wl.normal_velocity(wr, s, w.n_groups * w.rows_before(s), device=dev)
+            for s in range(w.n_steps)]
+    torch.cuda.synchronize()
+
+    def one_rollout(trace=None):
+        return ro.run(x0, w.step_coef, w.preview_coef, lambda s, x: vels[s], trace=trace)
+
+    for _ in range(max(args.warmup, 3)):
+        one_rollout()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.3)
+    traces = []
+    launches0 = B.launch_count()
+    torch.cuda.synchronize()
+    t_wall0 = time.time()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        tr = []
+        one_rollout(trace=tr)
+        traces.append(tr)
+    ev1.record()
+    torch.cuda.synchronize()
+    t_wall1 = time.time()
+    launches = B.launch_count() - launches0
+    clocks = sampler.stop(t_wall0, t_wall1)
+    total_ms = ev0.elapsed_time(ev1)
+    if dist is not None:
+        dist.barrier()
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+
+    # per-kernel device times from the events recorded inside the timed region
+    kinds = {}
+    for tr in traces:
+        for kind, rows, a, b in tr:
+            d = kinds.setdefault(kind, {"ms": 0.0, "rows": 0, "launches": 0})
+            d["ms"] += a.elapsed_time(b)
+            d["rows"] += rows
+            d["launches"] += 1
+    vel_bytes = 2 if w.vel_dtype == "bf16" else 4
+    step_bytes = kinds["step"]["rows"] * (w.elems * (8 + vel_bytes) + 4)
+    step_gbs = step_bytes / (kinds["step"]["ms"] * 1e-3) / 1e9
+    score_gbs, score_bytes = None, 0
+    if "score" in kinds:
+        score_bytes = kinds["score"]["rows"] * (w.elems * (4 + vel_bytes) + 4)
+        score_gbs = score_bytes / (kinds["score"]["ms"] * 1e-3) / 1e9
+    prune_stage_gbs = None
+    if "score" in kinds and "prune" in kinds:
+        ms = kinds["score"]["ms"] + kinds["prune"]["ms"]
+        prune_stage_gbs = (score_bytes + kinds["prune"]["rows"] * 8) / (ms * 1e-3) / 1e9
+    peak, peak_kind = _peaks()
+
+    # OVF selection microbenchmark (4096 groups x 256 scores -> 32) on rank 0
+    ovf = None
+    if rank == 0:
+        m = wl.OVF_MICRO
+        sc = torch.from_numpy(wl.ovf_micro_scores()).to(dev)
+        keep = torch.empty(m["n_groups"] * m["k"], dtype=torch.int32, device=dev)
+        kept = torch.empty(m["n_groups"] * m["k"], device=dev)
+        adv = torch.empty(m["n_groups"] * m["k"], device=dev)
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        best = []
+        for i in range(13):
+            flush.zero_()                       # evict the scores from L2 between repetitions
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            B.ovf_select_batched(m["n_groups"], m["n"], m["k"], sc, keep, kept, adv, 1e-6)
+            b.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                best.append(a.elapsed_time(b))
+        best.sort()
+        med = best[len(best) // 2]
+        ovf = {"groups_per_s": m["n_groups"] / (med * 1e-3), "us_per_launch": med * 1e3,
+               "workload": f"{m['n_groups']} groups x {m['n']} scores -> {m['k']} (select + index/score "
+                           "compaction + advantages), L2 flushed between repetitions"}
+
+    # end to end through the host-buffer entry point (pinned host memory, copies inside the timing)
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(B, wl, w, wr, rank, dist, dev, args)
+
+    value = world * w.traj_steps * args.steps / (total_ms * 1e-3)
+    if rank == 0:
+        line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": total_ms / args.steps,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+                "data": "synthetic", "config": _config(w, args), "clocks": clocks,
+                "gpu_launches": int(launches),
+                "roofline": {"bound": "hbm", "kernel": "step_kernel<bf16> (SDE step + log-prob)",
+                             "achieved": step_gbs, "peak": peak, "unit": "GB/s",
+                             "frac": step_gbs / peak, "peak_kind": peak_kind,
+                             "frac_of_8TBs_nominal": step_gbs / 8000.0, "traffic": None,
+                             "bytes_per_element_step": 8 + vel_bytes},
+                "kernels": {k: {"ms_per_rollout": v["ms"] / args.steps, "launches_per_rollout":
+                                v["launches"] // args.steps} for k, v in kinds.items()},
+                "score_gbs": score_gbs, "prune_stage_gbs": prune_stage_gbs,
+                "hbm_gbs_whole_rollout": (step_bytes + (score_bytes if score_gbs else 0)) / (total_ms * 1e-3) / 1e9,
+                "ovf_microbench": ovf, "e2e": e2e, "cpu_baseline": cpu_base}
+        print(json.dumps(line))
+    ro.close()
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+def run_e2e(B, wl, w, wr, rank, dist, dev, args):
+    import torch
+    cfg = B.make_config(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed,
+                        B.VEL_BF16 if w.vel_dtype == "bf16" else B.VEL_F32, adv_eps=w.adv_eps,
+                        group_offset=rank * w.n_groups)
+    ws = torch.empty(B.rollout_host_workspace_bytes(cfg), dtype=torch.uint8, device=dev)
+    dt = torch.bfloat16 if w.vel_dtype == "bf16" else torch.float32
+    # host inputs: pinned; filled from a seeded CPU generator block by block (content does not
+    # affect timing, but the bytes are real N(0,1) draws)
+    g = torch.Generator().manual_seed(1234 + rank)
+    x0 = torch.empty(w.n_groups * w.n_expand, w.elems, dtype=torch.float32).pin_memory()
+    block = torch.randn(64, w.elems, generator=g)
+    for i in range(0, x0.shape[0], 64):
+        x0[i:i + 64] = block[: x0.shape[0] - i].roll(i // 64, 1)
+    vels = []
+    vblock = torch.randn(64, w.elems, generator=g).to(dt)
+    for s in range(w.n_steps):
+        rows = w.n_groups * w.rows_before(s)
+        v = torch.empty(rows, w.elems, dtype=dt).pin_memory()
+        for i in range(0, rows, 64):
+            v[i:i + 64] = vblock[: rows - i].roll(s * 64 + i // 64, 1)
+        vels.append(v)
+    K = w.final_keep
+    x_final = torch.empty(w.n_groups * K, w.elems).pin_memory()
+    logp = torch.empty(w.traj_steps).pin_memory()
+    keep = torch.empty(sum(w.n_groups * k for _, k in w.stages), dtype=torch.int32).pin_memory()
+    adv = torch.empty(w.n_groups * K).pin_memory()
+    ids = torch.empty(w.n_groups * K, dtype=torch.int32).pin_memory()
+    coefs = [w.step_coef(s) for s in range(w.n_steps)]
+    pcoefs = [w.preview_coef(s) for s, _ in w.stages]
+
+    def call():
+        B.rollout_host(cfg, coefs, pcoefs, x0, vels, None, None, x_final, logp, keep, adv, ids, ws)
+
+    call()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    n = max(1, min(args.steps, 3))
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(n):
+        call()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b)
+    if dist is not None:
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    world = 1 if dist is None else dist.get_world_size()
+    h2d = x0.numel() * 4 + sum(v.numel() * v.element_size() for v in vels)
+    d2h = x_final.numel() * 4 + logp.numel() * 4 + keep.numel() * 4 + adv.numel() * 4 + ids.numel() * 4
+    return {"value": world * w.traj_steps * n / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": ms / n, "steps": n,
+            "entry": "pg_rollout_host (pinned host buffers, copies overlap compute)"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="large", choices=["large", "sd15", "tiny"])
+    ap.add_argument("--groups", type=int, default=0,
+                    help="prompt groups per GPU (default: the workload's own; smaller for profiling)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -47,6 +47,7 @@ class Rollout:
         self.x = [torch.empty(rows, elems, device=dev, dtype=torch.float32) for _ in range(2)]
         self.cur = 0
         self.k_cur = n_expand
+        self.trace = None
         self.scores = torch.empty(rows, device=dev, dtype=torch.float32)
         self.src_rows = torch.empty(rows, device=dev, dtype=torch.int32)
         self.rewards = torch.empty(rows, device=dev, dtype=torch.float32)
@@ -82,14 +83,22 @@ class Rollout:
     def n_active(self) -> int:
         return self.G * self.k_cur
 
-    def x_active(self) -> torch.Tensor:
-        return self.x[self.cur][: self.n_active]
-
-    def reset(self, x0: torch.Tensor):
+    def reset(self):
         B.rollout_reset(self.h)
         self.cur = 0
         self.k_cur = self.N0
-        self.x[0].copy_(x0)
+
+    def _timed(self, kind: str, rows: int, fn):
+        """Runs one library call, bracketed by CUDA events when tracing is on."""
+        if self.trace is None:
+            fn()
+            return
+        a = torch.cuda.Event(enable_timing=True)
+        b = torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        self.trace.append((kind, rows, a, b))
 
     def run(self, x0: torch.Tensor,
             step_coef: Callable[[int], Tuple[float, float, float]],
@@ -97,36 +106,45 @@ class Rollout:
             velocity: Callable[[int, torch.Tensor], torch.Tensor],
             external_scores: Optional[Callable[[int], torch.Tensor]] = None,
             final_rewards: Optional[Callable[[], torch.Tensor]] = None,
-            record_scores: bool = False) -> RolloutOutput:
+            record_scores: bool = False, trace: Optional[list] = None) -> RolloutOutput:
         """Runs the whole schedule.  ``velocity(step, x_active)`` returns the prediction for the
         currently active rows; ``external_scores(stage)`` / ``final_rewards()`` return device
-        fp32 tensors when the scores come from outside (else the preview mean / latent mean)."""
-        self.reset(x0)
+        fp32 tensors when the scores come from outside (else the preview mean / latent mean).
+        x0 is only read (step 0 writes into the driver's own buffer).  With ``trace`` (a list),
+        every library call is bracketed by CUDA events: (kind, rows, start, end) is appended."""
+        self.reset()
+        self.trace = trace
         out = RolloutOutput(x_final=None, logp=[], traj_id=None)
         stage_i, off = 0, 0
+        x_cur = x0                      # current latent tensor (x0 first, then own buffers)
         for s in range(self.T):
-            vel = velocity(s, self.x_active())
+            vel = velocity(s, x_cur[: self.n_active])
             src = None
             if stage_i < len(self.stages) and self.stages[stage_i][0] == s:
                 if external_scores is not None:
                     sc = external_scores(stage_i)
                 else:
                     sc = self.scores[: self.n_active]
-                    B.score(self.h, preview_coef(s), self.x[self.cur], vel, sc)
+                    self._timed("score", self.n_active, lambda: B.score(
+                        self.h, preview_coef(s), x_cur, vel, sc))
                 if record_scores:
                     out.stage_scores.append(sc.clone())
-                B.prune_ovf(self.h, stage_i, sc, self.keep[stage_i], self.src_rows,
-                            self.sel_var[stage_i])
+                self._timed("prune", self.n_active, lambda: B.prune_ovf(
+                    self.h, stage_i, sc, self.keep[stage_i], self.src_rows, self.sel_var[stage_i]))
                 self.k_cur = self.stages[stage_i][1]
                 src = self.src_rows
                 stage_i += 1
             rows = self.n_active
             lp = self.logp_all[off: off + rows]
-            if src is not None:
-                B.step(self.h, s, step_coef(s), self.x[self.cur], vel, src, self.x[self.cur ^ 1], lp)
-                self.cur ^= 1
+            if src is not None or x_cur is x0:
+                dst = self.x[self.cur ^ 1] if x_cur is self.x[self.cur] else self.x[self.cur]
             else:
-                B.step(self.h, s, step_coef(s), self.x[self.cur], vel, None, self.x[self.cur], lp)
+                dst = x_cur                                 # in place
+            self._timed("step", rows, lambda: B.step(self.h, s, step_coef(s), x_cur, vel, src, dst, lp))
+            if dst is not x_cur:
+                if x_cur is not x0:
+                    self.cur ^= 1
+                x_cur = dst
             out.logp.append(lp)
             off += rows
         rows = self.n_active
@@ -134,12 +152,13 @@ class Rollout:
             rw = final_rewards()
         else:
             rw = self.rewards[:rows]
-            B.score(self.h, (1.0, 0.0), self.x[self.cur], None, rw)
-        B.advantages(self.h, rw, self.adv, self.mean, self.std)
+            self._timed("reward", rows, lambda: B.score(self.h, (1.0, 0.0), x_cur, None, rw))
+        self._timed("advantages", rows, lambda: B.advantages(self.h, rw, self.adv, self.mean, self.std))
         ids = torch.empty(rows, device=self.dev, dtype=torch.int32)
         B.rollout_traj_ids(self.h, ids)
-        out.x_final = self.x_active()
+        out.x_final = x_cur[:rows]
         out.traj_id = ids
+        self.trace = None
         out.stage_keep = list(self.keep)
         out.stage_var = list(self.sel_var)
         out.rewards, out.adv, out.mean, out.std = rw, self.adv, self.mean, self.std

@@ -51,7 +51,7 @@ def test_normals_match_oracle(B):
         ref = oracle.normal_row(seed, step, int(t), d)
         worst = max(worst, np.abs(got[i] - ref).max())
     # fp32 hardware log2 / sin / cos against fp64: a few ulp of 1 in absolute terms
-    assert worst <= 2e-6, worst
+    assert worst <= 3e-6, worst
 
 
 # ------------------------------------------------------------------ step
