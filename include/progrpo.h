@@ -54,6 +54,7 @@ extern "C" {
 #define PG_ENONFINITE (-4)  /* reported by pg_rollout_status(): non-finite scores seen */
 #define PG_ETIMEOUT   (-5)  /* reported by pg_rollout_status(): a bounded device wait expired */
 #define PG_ENOMEM     (-6)  /* host or device allocation for the handle failed         */
+#define PG_ECAPACITY  (-7)  /* request larger than a fixed built-in buffer (pg_score_static) */
 
 #define PG_VEL_F32  0
 #define PG_VEL_BF16 1
@@ -219,6 +220,36 @@ int pg_rollout_host(const pg_config *cfg, const pg_step_coef *step_coef,
                     const void *const *vel_steps, const float *const *stage_scores,
                     const float *final_rewards, float *x_final, float *logp, int32_t *keep_idx,
                     float *adv, int32_t *traj_id, void *workspace, size_t workspace_bytes);
+
+/*
+ * Latent score without any allocation (no counterpart in the paper: this is a packaging
+ * variant of pg_score for restricted callers; the arithmetic is that of pg_score).
+ *
+ * For callers that cannot allocate device memory when they need a score: plug-ins running
+ * inside another framework's memory pool, services whose device footprint is fixed at
+ * start-up, code in a latency-critical section where cudaMalloc (which may synchronise the
+ * device) is unwelcome.  pg_score needs a handle and pg_rollout_init allocates; this call
+ * needs neither.  Its reduction scratch is a fixed array inside the library image
+ * (about 1 MB, resident on every GPU that loads the library until the process exits).
+ *
+ *   scores_out[i] = mean_e(p_x * x[i][e] + p_v * vel[i][e]),  i < n_rows
+ *   x [n_rows, elems] fp32, vel [n_rows, elems] fp32 or bf16 per vel_dtype (not read and may
+ *   be NULL when p_v == 0), scores_out [n_rows] fp32: caller-owned device memory, x and vel
+ *   16-byte aligned.  elems a positive multiple of 4.
+ *
+ * Limits: n_rows <= PG_STATIC_MAX_ROWS and n_rows * ceil(elems / 8192) <=
+ * PG_STATIC_MAX_PARTIALS; beyond either the call returns PG_ECAPACITY and does nothing
+ * (split the rows over several calls).  Calls no cudaMalloc / cudaFree.  The first call on
+ * each device looks up the device address of the built-in array; make that first call
+ * outside any stream capture.  All calls on a device share the array and it keeps the last
+ * call's contents (the call clears the counters it needs in stream order), so two calls
+ * whose kernels can overlap on the GPU (different streams, no ordering) race: keep calls
+ * on one stream or order them with events.
+ */
+#define PG_STATIC_MAX_ROWS     8192
+#define PG_STATIC_MAX_PARTIALS 262144
+int pg_score_static(int32_t n_rows, int32_t elems, int32_t vel_dtype, const pg_preview_coef *coef,
+                    const float *x, const void *vel, float *scores_out, void *stream);
 
 /* Copies the handle's current trajectory-id map ([n_active] int32, device
  * memory) to `dst` (device) in stream order. */

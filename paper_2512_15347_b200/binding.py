@@ -14,7 +14,8 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libprogrpo.so")
 
-OK, EINVAL, ESTATE, ECUDA, ENONFINITE, ETIMEOUT, ENOMEM = 0, -1, -2, -3, -4, -5, -6
+OK, EINVAL, ESTATE, ECUDA, ENONFINITE, ETIMEOUT, ENOMEM, ECAPACITY = 0, -1, -2, -3, -4, -5, -6, -7
+STATIC_MAX_ROWS, STATIC_MAX_PARTIALS = 8192, 262144
 VEL_F32, VEL_BF16 = 0, 1
 MAX_GROUP = 1024
 
@@ -75,6 +76,7 @@ def lib() -> ctypes.CDLL:
     L.pg_rollout_host.argtypes = [ctypes.POINTER(Config), ctypes.POINTER(StepCoef),
                                   ctypes.POINTER(PreviewCoef), vp, ctypes.POINTER(vp),
                                   ctypes.POINTER(vp), vp, vp, vp, vp, vp, vp, vp, sz]
+    L.pg_score_static.argtypes = [i32, i32, i32, ctypes.POINTER(PreviewCoef), vp, vp, vp, vp]
     L.pg_rollout_traj_ids.argtypes = [vp, vp, vp]
     L.pg_philox_raw.argtypes = [i64, vp, vp, vp, vp]
     L.pg_normal_rows.argtypes = [u64, i32, i32, i32, i32, vp, vp, vp]
@@ -85,7 +87,7 @@ def lib() -> ctypes.CDLL:
     for name in ("pg_rollout_init", "pg_rollout_destroy", "pg_rollout_reset", "pg_rollout_status",
                  "pg_step", "pg_score", "pg_prune_ovf", "pg_compact", "pg_advantages",
                  "pg_ovf_select_batched", "pg_rollout_host", "pg_rollout_traj_ids",
-                 "pg_philox_raw", "pg_normal_rows"):
+                 "pg_philox_raw", "pg_normal_rows", "pg_score_static"):
         getattr(L, name).restype = ctypes.c_int
     _lib = L
     return L
@@ -184,6 +186,14 @@ def ovf_select_batched(n_groups: int, n: int, k: int, scores, keep_idx, kept_sco
     _check(lib().pg_ovf_select_batched(n_groups, n, k, _p(scores), _p(keep_idx), _p(kept_scores),
                                        _p(adv), adv_eps, _p(status), _stream(stream)),
            "pg_ovf_select_batched")
+
+
+def score_static(n_rows: int, elems: int, vel_dtype: int, coef, x, vel, scores_out, stream=None) -> None:
+    """pg_score without a handle and without any allocation: the reduction scratch is a fixed
+    array inside the library (see pg_score_static for its limits and sharing rules)."""
+    c = PreviewCoef(*coef)
+    _check(lib().pg_score_static(n_rows, elems, vel_dtype, ctypes.byref(c), _p(x), _p(vel),
+                                 _p(scores_out), _stream(stream)), "pg_score_static")
 
 
 def rollout_traj_ids(h: int, dst, stream=None) -> None:

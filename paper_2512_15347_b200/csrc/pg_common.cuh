@@ -110,6 +110,8 @@ constexpr int kQuadsPerThread = 8;     // 4-element quads per thread and CTA
 constexpr int kChunkQuads = kRowThreads * kQuadsPerThread;   // 2048 quads = 8192 elements
 
 inline int chunks_per_row(int elems) { return (elems / 4 + kChunkQuads - 1) / kChunkQuads; }
+// partial sums per row that launch_score needs in RowScratch::partials
+inline int score_partials_per_row(int elems) { return chunks_per_row(elems); }
 
 // ---------------------------------------------------------------- launchers (device pointers)
 struct RowScratch {

@@ -246,6 +246,7 @@ const char* pg_strerror(int code) {
     case PG_ENONFINITE: return "non-finite scores were seen by the selection";
     case PG_ETIMEOUT: return "a bounded device-side wait expired";
     case PG_ENOMEM: return "out of memory";
+    case PG_ECAPACITY: return "request exceeds the capacity of a fixed built-in buffer";
     default: return "unknown error code";
   }
 }
