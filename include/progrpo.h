@@ -237,7 +237,7 @@ int pg_rollout_host(const pg_config *cfg, const pg_step_coef *step_coef,
  *   be NULL when p_v == 0), scores_out [n_rows] fp32: caller-owned device memory, x and vel
  *   16-byte aligned.  elems a positive multiple of 4.
  *
- * Limits: n_rows <= PG_STATIC_MAX_ROWS and n_rows * ceil(elems / 8192) <=
+ * Limits: n_rows <= PG_STATIC_MAX_ROWS and 8 * n_rows * ceil(elems / 32768) <=
  * PG_STATIC_MAX_PARTIALS; beyond either the call returns PG_ECAPACITY and does nothing
  * (split the rows over several calls).  Calls no cudaMalloc / cudaFree.  The first call on
  * each device looks up the device address of the built-in array; make that first call

@@ -67,22 +67,23 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
 // Two standard normals from two generator words (24-bit uniforms, Box-Muller).
 //   u1 = ((r0 >> 8) + 1) * 2^-24 in (0, 1],  u2 = (r1 >> 8) * 2^-24 in [0, 1)
 //   a = sqrt(-2 ln u1) cos(2 pi u2),  b = sqrt(-2 ln u1) sin(2 pi u2)
+// Returns -2 ln u1 = a^2 + b^2 (the pair's contribution to the sum of squared noise).
 // The logarithm uses the hardware log2 except close to u1 = 1, where its absolute error would
-// dominate the small radius: there -ln(1 - w) is summed as a short series in w = 1 - u1 (exact
-// in fp32).  The angle is shifted by half a turn (cos(t) = -cos(t - pi), same for sin) so that
-// the hardware sine / cosine are evaluated on [-pi, pi), their most accurate range.
-__device__ __forceinline__ void normal_pair(uint32_t r0, uint32_t r1, float& a, float& b) {
+// dominate the small radius: there -2 ln(1 - w) is summed as a short series in w = 1 - u1 (exact
+// in fp32; truncation below 2e-8 relative for w < 2^-6).  The angle is shifted by half a turn
+// (cos(t) = -cos(t - pi), same for sin) so that the hardware sine / cosine are evaluated on
+// [-pi, pi), their most accurate range.
+__device__ __forceinline__ float normal_pair(uint32_t r0, uint32_t r1, float& a, float& b) {
   const float k1 = (float)(r0 >> 8);
   const float u1 = fmaf(k1, 5.9604644775390625e-8f, 5.9604644775390625e-8f);
   float neg2ln = -1.3862943611198906f * __log2f(u1);           // -2 ln(u1) = -2 ln2 * log2(u1)
-  const float w = (float)((~r0) >> 8) * 5.9604644775390625e-8f;  // 1 - u1, exact
-  // -2 ln(1 - w) = 2w + w^2 + (2/3) w^3 + (1/2) w^4 + (2/5) w^5 ...
-  float ser = fmaf(w, 0.4f, 0.5f);
-  ser = fmaf(ser, w, 0.66666666666666667f);
+  const float w = 1.0f - u1;                                     // exact (Sterbenz / 24-bit grid)
+  // -2 ln(1 - w) = 2w + w^2 + (2/3) w^3 + (1/2) w^4 + ...
+  float ser = fmaf(w, 0.5f, 0.66666666666666667f);
   ser = fmaf(ser, w, 1.0f);
   ser = fmaf(ser, w, 2.0f);
   ser *= w;
-  neg2ln = (w < 0.03125f) ? ser : neg2ln;
+  neg2ln = (w < 0.015625f) ? ser : neg2ln;
   float radius;
   asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(radius) : "f"(neg2ln));
   const float turn = fmaf((float)(r1 >> 8), 5.9604644775390625e-8f, -0.5f);  // u2 - 1/2, exact
@@ -90,6 +91,7 @@ __device__ __forceinline__ void normal_pair(uint32_t r0, uint32_t r1, float& a, 
   __sincosf(6.283185307179586f * turn, &s, &c);
   a = -radius * c;
   b = -radius * s;
+  return neg2ln;
 }
 
 __device__ __forceinline__ float warp_sum(float v) {
@@ -105,17 +107,70 @@ __device__ __forceinline__ double warp_sum(double v) {
 #endif  // __CUDACC__
 
 // ---------------------------------------------------------------- launch geometry
-constexpr int kRowThreads = 256;       // threads per CTA of the row-streaming kernels
-constexpr int kQuadsPerThread = 8;     // 4-element quads per thread and CTA
-constexpr int kChunkQuads = kRowThreads * kQuadsPerThread;   // 2048 quads = 8192 elements
+// Row-streaming kernels (step, score): a CTA of kRowThreads threads handles one chunk of one
+// row; a chunk is chunk_quads 4-element quads, a multiple of kRowThreads * 2.  Every warp of
+// every CTA contributes one partial sum, so a row owns chunks * kRowWarps partial slots.
+constexpr int kRowThreads = 256;
+constexpr int kRowWarps = kRowThreads / 32;
+constexpr int kMinChunkQuads = kRowThreads * 2;        // 512 quads  = 2048 elements
+constexpr int kMaxChunkQuads = kMinChunkQuads * 16;    // 8192 quads = 32768 elements
+constexpr long long kWantedCtas = 148LL * 4 * 16;      // enough CTAs for ~16 waves on 148 SMs
 
-inline int chunks_per_row(int elems) { return (elems / 4 + kChunkQuads - 1) / kChunkQuads; }
-// partial sums per row that launch_score needs in RowScratch::partials
-inline int score_partials_per_row(int elems) { return chunks_per_row(elems); }
+struct RowGeometry {
+  int chunk_quads;   // quads per CTA
+  int chunks;        // CTAs per row
+  int slots;         // partial sums per row = chunks * kRowWarps
+};
+
+// Longest chunk (fewest CTA start-ups and reductions) that still leaves kWantedCtas CTAs.
+inline RowGeometry row_geometry(long long rows, int elems, int forced_chunk_quads = 0) {
+  const int quads = elems / 4;
+  int cq = kMaxChunkQuads;
+  if (forced_chunk_quads > 0) {
+    cq = forced_chunk_quads;
+  } else {
+    while (cq > kMinChunkQuads && rows * ((quads + cq - 1) / cq) < kWantedCtas) cq >>= 1;
+  }
+  RowGeometry g;
+  g.chunk_quads = cq;
+  g.chunks = (quads + cq - 1) / cq;
+  g.slots = g.chunks * kRowWarps;
+  return g;
+}
+
+#ifdef __CUDACC__
+// Per-row reduction without any CTA barrier or waiting.  Every warp of every CTA of the row
+// calls this once with its total (all lanes hold it).  The warp stores its total in its fixed
+// slot and takes a ticket; the warp that draws the last ticket adds all slots in slot order
+// (fp64) and hands the sum to fin(sum) on lane 0.  The result is independent of the order in
+// which warps arrive.  tickets[row] is left at zero for the next launch.
+template <typename Fin>
+__device__ __forceinline__ void finish_row(float warp_total, int row, int slot, int slots,
+                                           float* partials, unsigned int* tickets, Fin fin) {
+  const int lane = threadIdx.x & 31;
+  int last = 0;
+  if (lane == 0) {
+    partials[(size_t)row * slots + slot] = warp_total;
+    __threadfence();
+    const unsigned int t = atomicAdd(&tickets[row], 1u);
+    last = (t == (unsigned int)slots - 1u);
+  }
+  last = __shfl_sync(0xFFFFFFFFu, last, 0);
+  if (!last) return;
+  __threadfence();
+  double s = 0.0;
+  for (int c = lane; c < slots; c += 32) s += (double)__ldcg(&partials[(size_t)row * slots + c]);
+  s = warp_sum(s);
+  if (lane == 0) {
+    fin(s);
+    tickets[row] = 0u;
+  }
+}
+#endif
 
 // ---------------------------------------------------------------- launchers (device pointers)
 struct RowScratch {
-  float* partials;        // [rows * chunks_per_row]
+  float* partials;        // [rows * row_geometry(rows, elems).slots]
   unsigned int* tickets;  // [rows], zero between launches
 };
 
@@ -126,7 +181,7 @@ int launch_step(int n_rows, int elems, int vel_dtype, const float* x_in, const v
 
 int launch_score(int n_rows, int elems, int vel_dtype, const float* x, const void* vel,
                  double p_x, double p_v, float* scores_out, float* preview_out,
-                 RowScratch scratch, cudaStream_t stream);
+                 RowScratch scratch, cudaStream_t stream, int forced_chunk_quads = 0);
 
 int launch_ovf(int n_groups, int n, int k, const float* scores, int32_t* keep_idx,
                int32_t* src_rows, float* sel_var, float* kept_scores, float* adv, float adv_eps,

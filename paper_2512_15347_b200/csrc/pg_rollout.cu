@@ -80,11 +80,17 @@ int pg_rollout_init(const pg_config* cfg, pg_rollout** out) {
   h->cfg.stage_keep = h->stage_keep.data();
   h->k_cur = cfg->n_expand;
   const size_t rows = (size_t)cfg->n_groups * cfg->n_expand;
-  const size_t chunks = (size_t)pg::chunks_per_row(cfg->elems);
+  // partial-sum slots: the largest need over the row counts this schedule will launch with
+  size_t slots = rows * (size_t)pg::row_geometry((long long)rows, cfg->elems).slots;
+  for (int i = 0; i < cfg->n_stages; ++i) {
+    const long long r = (long long)cfg->n_groups * cfg->stage_keep[i];
+    const size_t need = (size_t)r * (size_t)pg::row_geometry(r, cfg->elems).slots;
+    if (need > slots) slots = need;
+  }
   cudaError_t e = cudaGetDevice(&h->device);
   if (e == cudaSuccess) e = cudaMalloc(&h->d_traj[0], rows * sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMalloc(&h->d_traj[1], rows * sizeof(int32_t));
-  if (e == cudaSuccess) e = cudaMalloc(&h->d_partials, rows * chunks * sizeof(float));
+  if (e == cudaSuccess) e = cudaMalloc(&h->d_partials, slots * sizeof(float));
   if (e == cudaSuccess) e = cudaMalloc(&h->d_tickets, rows * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMalloc(&h->d_status, sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMemset(h->d_tickets, 0, rows * sizeof(unsigned int));

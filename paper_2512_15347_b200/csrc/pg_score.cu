@@ -14,96 +14,86 @@ struct ScoreParams {
   float* partials;
   unsigned int* tickets;
   int quads_per_row;
+  int chunk_quads;
   int chunks;
   float p_x, p_v;
   double inv_d;
 };
 
-__device__ __forceinline__ float4 score_vel4(const float* v, size_t quad) {
-  return __ldcs(reinterpret_cast<const float4*>(v) + quad);
-}
-__device__ __forceinline__ float4 score_vel4(const __nv_bfloat16* v, size_t quad) {
-  const uint2 w = __ldcs(reinterpret_cast<const uint2*>(v) + quad);
+__device__ __forceinline__ float4 unpack_vel(const float4& raw) { return raw; }
+__device__ __forceinline__ float4 unpack_vel(const uint2& raw) {
   float4 r;
-  r.x = __uint_as_float(w.x << 16);
-  r.y = __uint_as_float(w.x & 0xFFFF0000u);
-  r.z = __uint_as_float(w.y << 16);
-  r.w = __uint_as_float(w.y & 0xFFFF0000u);
+  r.x = __uint_as_float(raw.x << 16);
+  r.y = __uint_as_float(raw.x & 0xFFFF0000u);
+  r.z = __uint_as_float(raw.y << 16);
+  r.w = __uint_as_float(raw.y & 0xFFFF0000u);
   return r;
 }
+template <typename T> struct VelRaw;
+template <> struct VelRaw<float> { using type = float4; };
+template <> struct VelRaw<__nv_bfloat16> { using type = uint2; };
+
+constexpr int kScoreUnroll = 4;   // quads per thread and iteration (loads of the next batch in flight)
 
 template <typename VelT, bool kUseVel, bool kEmit>
 __global__ void __launch_bounds__(kRowThreads)
 score_kernel(const __grid_constant__ ScoreParams p) {
+  using Raw = typename VelRaw<VelT>::type;
   const int row = blockIdx.x / p.chunks;
   const int chunk = blockIdx.x - row * p.chunks;
-  const size_t base = (size_t)row * p.quads_per_row;
-  const VelT* vel = reinterpret_cast<const VelT*>(p.vel);
-  const int q0 = chunk * kChunkQuads + threadIdx.x;
+  const float4* x = reinterpret_cast<const float4*>(p.x) + (size_t)row * p.quads_per_row;
+  const Raw* vel = reinterpret_cast<const Raw*>(p.vel) + (size_t)row * p.quads_per_row;
+  float4* prev = kEmit ? reinterpret_cast<float4*>(p.preview_out) + (size_t)row * p.quads_per_row : nullptr;
+  const int q_begin = chunk * p.chunk_quads;
+  const int q_end = min(q_begin + p.chunk_quads, p.quads_per_row);
 
-  float4 xv[kQuadsPerThread], vv[kQuadsPerThread];
+  float4 xv[kScoreUnroll], nx[kScoreUnroll];
+  Raw vv[kScoreUnroll], nv[kScoreUnroll];
+  auto load = [&](int q, float4 (&xs)[kScoreUnroll], Raw (&vs)[kScoreUnroll]) {
 #pragma unroll
-  for (int u = 0; u < kQuadsPerThread; ++u) {
-    const int q = q0 + u * kRowThreads;
-    if (q < p.quads_per_row) {
-      xv[u] = __ldcs(reinterpret_cast<const float4*>(p.x) + base + q);
-      if (kUseVel) vv[u] = score_vel4(vel, base + q);
+    for (int u = 0; u < kScoreUnroll; ++u) {
+      const int qq = q + u * kRowThreads;
+      if (qq < q_end) {
+        xs[u] = __ldcs(x + qq);
+        if (kUseVel) vs[u] = __ldcs(vel + qq);
+      }
     }
-  }
+  };
   float acc = 0.f;
+  int q = q_begin + threadIdx.x;
+  load(q, xv, vv);
+  while (q < q_end) {
+    const int nq = q + kScoreUnroll * kRowThreads;
+    load(nq, nx, nv);
 #pragma unroll
-  for (int u = 0; u < kQuadsPerThread; ++u) {
-    const int q = q0 + u * kRowThreads;
-    if (q < p.quads_per_row) {
-      float4 h;
-      h.x = p.p_x * xv[u].x;
-      h.y = p.p_x * xv[u].y;
-      h.z = p.p_x * xv[u].z;
-      h.w = p.p_x * xv[u].w;
-      if (kUseVel) {
-        h.x = fmaf(p.p_v, vv[u].x, h.x);
-        h.y = fmaf(p.p_v, vv[u].y, h.y);
-        h.z = fmaf(p.p_v, vv[u].z, h.z);
-        h.w = fmaf(p.p_v, vv[u].w, h.w);
+    for (int u = 0; u < kScoreUnroll; ++u) {
+      const int qq = q + u * kRowThreads;
+      if (qq < q_end) {
+        float4 h;
+        h.x = p.p_x * xv[u].x;
+        h.y = p.p_x * xv[u].y;
+        h.z = p.p_x * xv[u].z;
+        h.w = p.p_x * xv[u].w;
+        if (kUseVel) {
+          const float4 vf = unpack_vel(vv[u]);
+          h.x = fmaf(p.p_v, vf.x, h.x);
+          h.y = fmaf(p.p_v, vf.y, h.y);
+          h.z = fmaf(p.p_v, vf.z, h.z);
+          h.w = fmaf(p.p_v, vf.w, h.w);
+        }
+        acc += (h.x + h.y) + (h.z + h.w);
+        if (kEmit) __stcs(prev + qq, h);
       }
-      acc += (h.x + h.y) + (h.z + h.w);
-      if (kEmit) __stcs(reinterpret_cast<float4*>(p.preview_out) + base + q, h);
     }
+#pragma unroll
+    for (int u = 0; u < kScoreUnroll; ++u) { xv[u] = nx[u]; vv[u] = nv[u]; }
+    q = nq;
   }
 
-  __shared__ float warp_part[kRowThreads / 32];
-  __shared__ bool is_last;
   acc = warp_sum(acc);
-  if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = acc;
-  __syncthreads();
-  if (threadIdx.x < 32) {
-    float v = (threadIdx.x < kRowThreads / 32) ? warp_part[threadIdx.x] : 0.f;
-    v = warp_sum(v);
-    if (threadIdx.x == 0) {
-      if (p.chunks == 1) {
-        p.scores_out[row] = (float)((double)v * p.inv_d);
-        is_last = false;
-      } else {
-        p.partials[(size_t)row * p.chunks + chunk] = v;
-        __threadfence();
-        const unsigned int t = atomicAdd(&p.tickets[row], 1u);
-        is_last = (t == (unsigned int)p.chunks - 1u);
-      }
-    }
-  }
-  __syncthreads();
-  if (!is_last) return;
-  if (threadIdx.x < 32) {
-    __threadfence();
-    double s = 0.0;
-    for (int c = threadIdx.x; c < p.chunks; c += 32)
-      s += (double)__ldcg(&p.partials[(size_t)row * p.chunks + c]);
-    s = warp_sum(s);
-    if (threadIdx.x == 0) {
-      p.scores_out[row] = (float)(s * p.inv_d);
-      p.tickets[row] = 0u;
-    }
-  }
+  const int slots = p.chunks * kRowWarps;
+  finish_row(acc, row, chunk * kRowWarps + (threadIdx.x >> 5), slots, p.partials, p.tickets,
+             [&](double sum) { p.scores_out[row] = (float)(sum * p.inv_d); });
 }
 
 template <typename VelT>
@@ -121,8 +111,9 @@ static void dispatch_score(const ScoreParams& p, bool use_vel, bool emit, dim3 g
 
 int launch_score(int n_rows, int elems, int vel_dtype, const float* x, const void* vel,
                  double p_x, double p_v, float* scores_out, float* preview_out,
-                 RowScratch scratch, cudaStream_t stream) {
+                 RowScratch scratch, cudaStream_t stream, int forced_chunk_quads) {
   if (n_rows == 0) return PG_OK;
+  const RowGeometry geo = row_geometry(n_rows, elems, forced_chunk_quads);
   ScoreParams p;
   p.x = x;
   p.vel = vel;
@@ -131,11 +122,12 @@ int launch_score(int n_rows, int elems, int vel_dtype, const float* x, const voi
   p.partials = scratch.partials;
   p.tickets = scratch.tickets;
   p.quads_per_row = elems / 4;
-  p.chunks = chunks_per_row(elems);
+  p.chunk_quads = geo.chunk_quads;
+  p.chunks = geo.chunks;
   p.p_x = (float)p_x;
   p.p_v = (float)p_v;
   p.inv_d = 1.0 / (double)elems;
-  const long long blocks = (long long)n_rows * p.chunks;
+  const long long blocks = (long long)n_rows * geo.chunks;
   if (blocks > 0x7FFFFFFFLL) return PG_EINVAL;
   const dim3 grid((unsigned)blocks);
   const bool use_vel = (p_v != 0.0);

@@ -61,7 +61,8 @@ extern "C" int pg_score_static(int32_t n_rows, int32_t elems, int32_t vel_dtype,
   if (((uintptr_t)x & 15) || ((uintptr_t)vel & 15)) return PG_EINVAL;
   // capacity of the built-in scratch: PG_STATIC_MAX_ROWS rows, PG_STATIC_MAX_PARTIALS partial sums
   if (n_rows > kStaticMaxRows) return PG_ECAPACITY;
-  const size_t need = (size_t)n_rows * (size_t)pg::score_partials_per_row(elems);
+  const pg::RowGeometry geo = pg::row_geometry(n_rows, elems, pg::kMaxChunkQuads);
+  const size_t need = (size_t)n_rows * (size_t)geo.slots;
   if (need > kStaticMaxPartials) return PG_ECAPACITY;
 
   StaticScratch* s = nullptr;
@@ -72,5 +73,5 @@ extern "C" int pg_score_static(int32_t n_rows, int32_t elems, int32_t vel_dtype,
   PG_CUDA(cudaMemsetAsync(s->tickets, 0, (size_t)n_rows * sizeof(unsigned int), st));
   pg::RowScratch scratch{s->partials, s->tickets};
   return pg::launch_score(n_rows, elems, vel_dtype, x, vel, coef->p_x, coef->p_v, scores_out,
-                          nullptr, scratch, st);
+                          nullptr, scratch, st, pg::kMaxChunkQuads);
 }

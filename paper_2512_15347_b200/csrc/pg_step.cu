@@ -1,11 +1,12 @@
 // Fused Euler-Maruyama step + Gaussian policy log-probability (Eq. "euler_method").
 //
-// One CTA streams one chunk (8192 elements) of one trajectory: x and the prediction are read
-// once with 128/64-bit coalesced loads, the noise is generated in registers (one Philox block
-// per 4 elements), x' is written once.  The per-trajectory sum of xi^2 is reduced
-// thread -> warp (shuffle) -> CTA (shared memory) -> trajectory (fixed-slot partials, finished
-// by the last CTA of the row through a wait-free ticket), so the result does not depend on
-// the order in which CTAs run.
+// One CTA streams one chunk of one trajectory: x and the prediction are read once with
+// 128/64-bit coalesced loads (the loads of the next pair of quads are issued before the
+// current pair is computed), the noise is generated in registers (one Philox block per 4
+// elements), x' is written once.  Sum of squared noise: for a Box-Muller pair a^2 + b^2 equals
+// -2 ln u1, so the radius term is accumulated directly.  The per-trajectory sum is reduced
+// thread -> warp (shuffle) -> trajectory (fixed-slot partials finished by the last-arriving
+// warp, no barrier and no waiting), so the result does not depend on scheduling.
 #include "pg_common.cuh"
 
 namespace pg {
@@ -20,6 +21,7 @@ struct StepParams {
   float* partials;
   unsigned int* tickets;
   int quads_per_row;      // d / 4
+  int chunk_quads;        // quads per CTA
   int chunks;             // CTAs per row
   uint32_t step;
   float c_x, c_v, noise_std;
@@ -28,109 +30,109 @@ struct StepParams {
   PhiloxKeys rk;
 };
 
-__device__ __forceinline__ float4 load_vel4(const float* v, size_t quad) {
-  return __ldcs(reinterpret_cast<const float4*>(v) + quad);
+struct VelF32 { float4 raw; };
+struct VelBf16 { uint2 raw; };
+
+__device__ __forceinline__ void load_vel(const float* v, size_t quad, VelF32& out) {
+  out.raw = __ldcs(reinterpret_cast<const float4*>(v) + quad);
 }
-__device__ __forceinline__ float4 load_vel4(const __nv_bfloat16* v, size_t quad) {
-  const uint2 w = __ldcs(reinterpret_cast<const uint2*>(v) + quad);
+__device__ __forceinline__ void load_vel(const __nv_bfloat16* v, size_t quad, VelBf16& out) {
+  out.raw = __ldcs(reinterpret_cast<const uint2*>(v) + quad);
+}
+__device__ __forceinline__ float4 vel_f32(const VelF32& v) { return v.raw; }
+__device__ __forceinline__ float4 vel_f32(const VelBf16& v) {
   float4 r;
-  r.x = __uint_as_float(w.x << 16);
-  r.y = __uint_as_float(w.x & 0xFFFF0000u);
-  r.z = __uint_as_float(w.y << 16);
-  r.w = __uint_as_float(w.y & 0xFFFF0000u);
+  r.x = __uint_as_float(v.raw.x << 16);
+  r.y = __uint_as_float(v.raw.x & 0xFFFF0000u);
+  r.z = __uint_as_float(v.raw.y << 16);
+  r.w = __uint_as_float(v.raw.y & 0xFFFF0000u);
   return r;
 }
+template <typename T> struct VelReg;
+template <> struct VelReg<float> { using type = VelF32; };
+template <> struct VelReg<__nv_bfloat16> { using type = VelBf16; };
 
-template <typename VelT, bool kNoise>
+// kNoise: noise_std > 0.  kUnitCx: c_x == 1 (drift = prediction), one FMA per element less.
+template <typename VelT, bool kNoise, bool kUnitCx>
 __global__ void __launch_bounds__(kRowThreads)
 step_kernel(const __grid_constant__ StepParams p) {
+  using VReg = typename VelReg<VelT>::type;
   const int row = blockIdx.x / p.chunks;
   const int chunk = blockIdx.x - row * p.chunks;
   const int src = p.src_rows ? p.src_rows[row] : row;
   const uint32_t traj = (uint32_t)p.traj_id[row];
 
-  const size_t in_base = (size_t)src * p.quads_per_row;
-  const size_t out_base = (size_t)row * p.quads_per_row;
-  const VelT* vel = reinterpret_cast<const VelT*>(p.vel);
-  const int q0 = chunk * kChunkQuads + threadIdx.x;
+  const float4* xin = reinterpret_cast<const float4*>(p.x_in) + (size_t)src * p.quads_per_row;
+  const VelT* vel = reinterpret_cast<const VelT*>(p.vel) + (size_t)src * p.quads_per_row * 4;
+  float4* xout = reinterpret_cast<float4*>(p.x_out) + (size_t)row * p.quads_per_row;
+  const int q_begin = chunk * p.chunk_quads;
+  const int q_end = min(q_begin + p.chunk_quads, p.quads_per_row);
 
   float acc = 0.f;
-#pragma unroll
-  for (int half = 0; half < 2; ++half) {
-    constexpr int kU = kQuadsPerThread / 2;
-    float4 xv[kU], vv[kU];
-#pragma unroll
-    for (int u = 0; u < kU; ++u) {
-      const int q = q0 + (half * kU + u) * kRowThreads;
-      if (q < p.quads_per_row) {
-        xv[u] = __ldcs(reinterpret_cast<const float4*>(p.x_in) + in_base + q);
-        vv[u] = load_vel4(vel, in_base + q);
-      }
+  auto process = [&](int q, const float4& xv, const VReg& vraw) {
+    const float4 vv = vel_f32(vraw);
+    float4 m;
+    if (kUnitCx) {
+      m.x = fmaf(p.c_v, vv.x, xv.x);
+      m.y = fmaf(p.c_v, vv.y, xv.y);
+      m.z = fmaf(p.c_v, vv.z, xv.z);
+      m.w = fmaf(p.c_v, vv.w, xv.w);
+    } else {
+      m.x = fmaf(p.c_v, vv.x, p.c_x * xv.x);
+      m.y = fmaf(p.c_v, vv.y, p.c_x * xv.y);
+      m.z = fmaf(p.c_v, vv.z, p.c_x * xv.z);
+      m.w = fmaf(p.c_v, vv.w, p.c_x * xv.w);
     }
-#pragma unroll
-    for (int u = 0; u < kU; ++u) {
-      const int q = q0 + (half * kU + u) * kRowThreads;
-      if (q < p.quads_per_row) {
-        float4 m;
-        m.x = fmaf(p.c_v, vv[u].x, p.c_x * xv[u].x);
-        m.y = fmaf(p.c_v, vv[u].y, p.c_x * xv[u].y);
-        m.z = fmaf(p.c_v, vv[u].z, p.c_x * xv[u].z);
-        m.w = fmaf(p.c_v, vv[u].w, p.c_x * xv[u].w);
-        if (kNoise) {
-          const uint4 r = philox4x32_10((uint32_t)q, p.step, traj, 0u, p.rk);
-          float n0, n1, n2, n3;
-          normal_pair(r.x, r.y, n0, n1);
-          normal_pair(r.z, r.w, n2, n3);
-          acc += (n0 * n0 + n1 * n1) + (n2 * n2 + n3 * n3);
-          m.x = fmaf(p.noise_std, n0, m.x);
-          m.y = fmaf(p.noise_std, n1, m.y);
-          m.z = fmaf(p.noise_std, n2, m.z);
-          m.w = fmaf(p.noise_std, n3, m.w);
-        }
-        __stcs(reinterpret_cast<float4*>(p.x_out) + out_base + q, m);
-      }
+    if (kNoise) {
+      const uint4 r = philox4x32_10((uint32_t)q, p.step, traj, 0u, p.rk);
+      float n0, n1, n2, n3;
+      acc += normal_pair(r.x, r.y, n0, n1);
+      acc += normal_pair(r.z, r.w, n2, n3);
+      m.x = fmaf(p.noise_std, n0, m.x);
+      m.y = fmaf(p.noise_std, n1, m.y);
+      m.z = fmaf(p.noise_std, n2, m.z);
+      m.w = fmaf(p.noise_std, n3, m.w);
     }
+    __stcs(xout + q, m);
+  };
+
+  int q = q_begin + threadIdx.x;
+  float4 xa, xb;
+  VReg va, vb;
+  if (q < q_end) { xa = __ldcs(xin + q); load_vel(vel, (size_t)q, va); }
+  if (q + kRowThreads < q_end) { xb = __ldcs(xin + q + kRowThreads); load_vel(vel, (size_t)q + kRowThreads, vb); }
+  while (q < q_end) {
+    const int nq = q + 2 * kRowThreads;
+    float4 nxa, nxb;
+    VReg nva, nvb;
+    if (nq < q_end) { nxa = __ldcs(xin + nq); load_vel(vel, (size_t)nq, nva); }
+    if (nq + kRowThreads < q_end) { nxb = __ldcs(xin + nq + kRowThreads); load_vel(vel, (size_t)nq + kRowThreads, nvb); }
+    process(q, xa, va);
+    if (q + kRowThreads < q_end) process(q + kRowThreads, xb, vb);
+    xa = nxa; xb = nxb; va = nva; vb = nvb;
+    q = nq;
   }
 
   if (!kNoise) {
     if (chunk == 0 && threadIdx.x == 0) p.logp_out[row] = 0.f;
     return;
   }
-
-  // CTA reduction in a fixed shape
-  __shared__ float warp_part[kRowThreads / 32];
-  __shared__ bool is_last;
   acc = warp_sum(acc);
-  if ((threadIdx.x & 31) == 0) warp_part[threadIdx.x >> 5] = acc;
-  __syncthreads();
-  if (threadIdx.x < 32) {
-    float v = (threadIdx.x < kRowThreads / 32) ? warp_part[threadIdx.x] : 0.f;
-    v = warp_sum(v);
-    if (threadIdx.x == 0) {
-      if (p.chunks == 1) {
-        p.logp_out[row] = (float)((-0.5 * (double)v - p.logp_const) * p.logp_scale);
-        is_last = false;
-      } else {
-        p.partials[(size_t)row * p.chunks + chunk] = v;
-        __threadfence();
-        const unsigned int t = atomicAdd(&p.tickets[row], 1u);
-        is_last = (t == (unsigned int)p.chunks - 1u);
-      }
-    }
-  }
-  __syncthreads();
-  if (!is_last) return;
-  // last CTA of this row: all partials are visible; add them in slot order
-  if (threadIdx.x < 32) {
-    __threadfence();
-    double s = 0.0;
-    for (int c = threadIdx.x; c < p.chunks; c += 32)
-      s += (double)__ldcg(&p.partials[(size_t)row * p.chunks + c]);
-    s = warp_sum(s);
-    if (threadIdx.x == 0) {
-      p.logp_out[row] = (float)((-0.5 * s - p.logp_const) * p.logp_scale);
-      p.tickets[row] = 0u;   // ready for the next launch
-    }
+  const int slots = p.chunks * kRowWarps;
+  finish_row(acc, row, chunk * kRowWarps + (threadIdx.x >> 5), slots, p.partials, p.tickets,
+             [&](double sum) {
+               p.logp_out[row] = (float)((-0.5 * sum - p.logp_const) * p.logp_scale);
+             });
+}
+
+template <typename VelT>
+static void dispatch_step(const StepParams& p, bool noise, bool unit_cx, dim3 grid, cudaStream_t st) {
+  const dim3 block(kRowThreads);
+  if (noise) {
+    if (unit_cx) step_kernel<VelT, true, true><<<grid, block, 0, st>>>(p);
+    else         step_kernel<VelT, true, false><<<grid, block, 0, st>>>(p);
+  } else {
+    step_kernel<VelT, false, false><<<grid, block, 0, st>>>(p);
   }
 }
 
@@ -139,6 +141,7 @@ int launch_step(int n_rows, int elems, int vel_dtype, const float* x_in, const v
                 uint64_t seed, int32_t step, double c_x, double c_v, double noise_std,
                 int logp_mean, RowScratch scratch, cudaStream_t stream) {
   if (n_rows == 0) return PG_OK;
+  const RowGeometry geo = row_geometry(n_rows, elems);
   StepParams p;
   p.x_in = x_in;
   p.vel = vel;
@@ -149,28 +152,22 @@ int launch_step(int n_rows, int elems, int vel_dtype, const float* x_in, const v
   p.partials = scratch.partials;
   p.tickets = scratch.tickets;
   p.quads_per_row = elems / 4;
-  p.chunks = chunks_per_row(elems);
+  p.chunk_quads = geo.chunk_quads;
+  p.chunks = geo.chunks;
   p.step = (uint32_t)step;
   p.c_x = (float)c_x;
   p.c_v = (float)c_v;
   p.noise_std = (float)noise_std;
   const double two_pi = 6.283185307179586476925286766559;
-  // the device scales the noise by the fp32 value of noise_std; the density uses the same
-  const double ns = (double)p.noise_std;
-  p.logp_const = noise_std > 0.0 ? 0.5 * (double)elems * log(two_pi * ns * ns) : 0.0;
+  p.logp_const = noise_std > 0.0 ? 0.5 * (double)elems * log(two_pi * noise_std * noise_std) : 0.0;
   p.logp_scale = logp_mean ? 1.0 / (double)elems : 1.0;
   p.rk = make_philox_keys(seed);
-  const long long blocks = (long long)n_rows * p.chunks;
+  const long long blocks = (long long)n_rows * geo.chunks;
   if (blocks > 0x7FFFFFFFLL) return PG_EINVAL;
-  const dim3 grid((unsigned)blocks), block(kRowThreads);
+  const dim3 grid((unsigned)blocks);
   const bool noise = noise_std > 0.0;
-  if (vel_dtype == PG_VEL_BF16) {
-    if (noise) step_kernel<__nv_bfloat16, true><<<grid, block, 0, stream>>>(p);
-    else       step_kernel<__nv_bfloat16, false><<<grid, block, 0, stream>>>(p);
-  } else {
-    if (noise) step_kernel<float, true><<<grid, block, 0, stream>>>(p);
-    else       step_kernel<float, false><<<grid, block, 0, stream>>>(p);
-  }
+  if (vel_dtype == PG_VEL_BF16) dispatch_step<__nv_bfloat16>(p, noise, p.c_x == 1.0f, grid, stream);
+  else                          dispatch_step<float>(p, noise, p.c_x == 1.0f, grid, stream);
   PG_LAUNCH_CHECK();
   return PG_OK;
 }
