@@ -244,6 +244,215 @@ ovf_select_kernel(const __grid_constant__ OvfParams p) {
   }
 }
 
+// ---------------------------------------------------------------- groups of up to 256 scores
+//
+// One warp per group, E = 1, 2, 4 or 8 scores per lane (n <= 32 * E).  The 64-bit keys are
+// sorted with a bitonic network held in registers (exchanges inside a lane for distances
+// below E, warp shuffles above); slots >= n hold an all-ones key and sort to the end.  Since
+// keys are distinct any correct sorting network yields the same order as the counting kernel.
+// No CTA barrier is used: warps of a CTA are independent.
+constexpr int kOvfWarpsPerCta = 4;
+
+__device__ __forceinline__ float key_to_score(uint32_t key) {
+  const uint32_t b = (key & 0x80000000u) ? (key ^ 0x80000000u) : ~key;
+  return __uint_as_float(b);      // all-ones key -> 0x7FFFFFFF, a NaN, as it went in
+}
+
+template <int E>
+__global__ void __launch_bounds__(kOvfWarpsPerCta * 32)
+ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
+  constexpr int N = 32 * E;
+  extern __shared__ __align__(16) unsigned char smem[];
+  const int n = p.n, k = p.k;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int g = blockIdx.x * kOvfWarpsPerCta + warp;
+  if (g >= n_groups) return;
+  const size_t per_warp = (size_t)(k + 1) * 4 * sizeof(double) + (size_t)N * sizeof(float) + 32;
+  unsigned char* base = smem + (size_t)warp * per_warp;
+  double* L1 = reinterpret_cast<double*>(base);
+  double* L2 = L1 + (k + 1);
+  double* H1 = L2 + (k + 1);
+  double* H2 = H1 + (k + 1);
+  float* sorted = reinterpret_cast<float*>(H2 + (k + 1));
+  unsigned int* mask = reinterpret_cast<unsigned int*>(sorted + N);     // N bits, 8 words
+
+  const float* sc = p.scores + (size_t)g * n;
+  float orig[E];
+  unsigned long long key[E];
+  bool bad = false;
+#pragma unroll
+  for (int r = 0; r < E; ++r) {
+    const int i = lane * E + r;
+    if (i < n) {
+      orig[r] = sc[i];
+      bad |= !(fabsf(orig[r]) <= FLT_MAX);
+      key[r] = ((unsigned long long)order_key(orig[r]) << 32) | (unsigned int)i;
+    } else {
+      orig[r] = 0.f;
+      key[r] = ~0ull;
+    }
+  }
+  if (bad && p.status) atomicOr(p.status, 1);
+  if (lane < 8) mask[lane] = 0u;
+
+  // Bitonic sort, ascending over index lane * E + r, in the form whose compare-exchanges all
+  // point the same way: each merge of two sorted runs of length size/2 first pairs i with its
+  // mirror i ^ (size - 1), then halves the distance; the lower index always keeps the minimum.
+#pragma unroll
+  for (int size = 2; size <= N; size <<= 1) {
+    // mirror step
+    if (size <= E) {
+#pragma unroll
+      for (int r = 0; r < E; ++r) {
+        const int q = r ^ (size - 1);
+        if (r < q) {
+          const unsigned long long a = key[r], b = key[q];
+          const bool swap = a > b;
+          key[r] = swap ? b : a;
+          key[q] = swap ? a : b;
+        }
+      }
+    } else {
+      const int lane_mask = size / E - 1;
+      const bool lower = (lane & (size / E / 2)) == 0;
+      unsigned long long other[E];
+#pragma unroll
+      for (int r = 0; r < E; ++r) other[r] = __shfl_xor_sync(0xFFFFFFFFu, key[r ^ (E - 1)], lane_mask);
+#pragma unroll
+      for (int r = 0; r < E; ++r) {
+        const bool other_smaller = other[r] < key[r];
+        key[r] = (lower == other_smaller) ? other[r] : key[r];
+      }
+    }
+    // halving steps
+#pragma unroll
+    for (int j = size >> 2; j > 0; j >>= 1) {
+      if (j < E) {
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+          if ((r & j) == 0) {
+            const unsigned long long a = key[r], b = key[r | j];
+            const bool swap = a > b;
+            key[r] = swap ? b : a;
+            key[r | j] = swap ? a : b;
+          }
+        }
+      } else {
+        const int lane_mask = j / E;
+        const bool lower = (lane & lane_mask) == 0;
+#pragma unroll
+        for (int r = 0; r < E; ++r) {
+          const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, key[r], lane_mask);
+          const bool other_smaller = other < key[r];
+          key[r] = (lower == other_smaller) ? other : key[r];
+        }
+      }
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < E; ++r) sorted[lane * E + r] = key_to_score((uint32_t)(key[r] >> 32));
+  __syncwarp();
+
+  // running sums from both ends, serial and in order (fp64, explicitly rounded)
+  if (lane < 2) {
+    const double pivot = arithmetic_value(sorted[n / 2]);
+    double a1 = 0.0, a2 = 0.0;
+    double* S1 = lane == 0 ? L1 : H1;
+    double* S2 = lane == 0 ? L2 : H2;
+    S1[0] = 0.0;
+    S2[0] = 0.0;
+    for (int j = 1; j <= k; ++j) {
+      const int pos = lane == 0 ? (j - 1) : (n - j);
+      const double c = __dsub_rn(arithmetic_value(sorted[pos]), pivot);
+      a1 = __dadd_rn(a1, c);
+      a2 = __dadd_rn(a2, __dmul_rn(c, c));
+      S1[j] = a1;
+      S2[j] = a2;
+    }
+  }
+  __syncwarp();
+
+  double best_m = -1.0;
+  int best_j = -1;
+  for (int j = lane; j <= k; j += 32) {
+    const double S = __dadd_rn(L1[j], H1[k - j]);
+    const double Q = __dadd_rn(L2[j], H2[k - j]);
+    const double M = __dsub_rn(__dmul_rn((double)k, Q), __dmul_rn(S, S));
+    if (best_j < 0 || M >= best_m) { best_m = M; best_j = j; }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const double om = __shfl_xor_sync(0xFFFFFFFFu, best_m, o);
+    const int oj = __shfl_xor_sync(0xFFFFFFFFu, best_j, o);
+    if (oj >= 0 && (best_j < 0 || om > best_m || (om == best_m && oj > best_j))) {
+      best_m = om; best_j = oj;
+    }
+  }
+  const int jstar = best_j;
+  const int high_from = n - (k - jstar);
+  if (lane == 0 && p.sel_var) p.sel_var[g] = (float)(best_m / ((double)k * (double)k));
+
+  // kept slots as a bit set, then ascending slot order by popcount prefix
+#pragma unroll
+  for (int r = 0; r < E; ++r) {
+    const int pos = lane * E + r;
+    if (pos < n && (pos < jstar || pos >= high_from)) {
+      const unsigned int slot = (unsigned int)key[r];
+      atomicOr(&mask[slot >> 5], 1u << (slot & 31));
+    }
+  }
+  __syncwarp();
+  const int first = lane * E;
+  const unsigned int bits = (mask[first >> 5] >> (first & 31)) & ((E == 32) ? 0xFFFFFFFFu : ((1u << E) - 1u));
+  const int cnt = __popc(bits);
+  int incl = cnt;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  int pos = incl - cnt;
+  double sum_kept = 0.0;
+#pragma unroll
+  for (int r = 0; r < E; ++r) {
+    if (bits & (1u << r)) {
+      const int i = first + r;
+      const size_t o = (size_t)g * k + pos;
+      p.keep_idx[o] = i;
+      if (p.src_rows) p.src_rows[o] = g * n + i;
+      if (p.traj_out) p.traj_out[o] = p.traj_in[(size_t)g * n + i];
+      if (p.kept_scores) p.kept_scores[o] = orig[r];
+      sum_kept += (double)orig[r];
+      ++pos;
+    }
+  }
+  if (p.adv) {
+    const double mu = warp_sum(sum_kept) / (double)k;
+    double sq = 0.0;
+#pragma unroll
+    for (int r = 0; r < E; ++r)
+      if (bits & (1u << r)) {
+        const double dlt = (double)orig[r] - mu;
+        sq += dlt * dlt;
+      }
+    const double denom = sqrt(warp_sum(sq) / (double)k) + (double)p.adv_eps;
+    pos = incl - cnt;
+#pragma unroll
+    for (int r = 0; r < E; ++r)
+      if (bits & (1u << r)) {
+        p.adv[(size_t)g * k + pos] = (float)(((double)orig[r] - mu) / denom);
+        ++pos;
+      }
+  }
+}
+
+template <int E>
+static void launch_ovf_warp(const OvfParams& p, int n_groups, cudaStream_t stream) {
+  const size_t per_warp = (size_t)(p.k + 1) * 4 * sizeof(double) + (size_t)(32 * E) * sizeof(float) + 32;
+  const int ctas = (n_groups + kOvfWarpsPerCta - 1) / kOvfWarpsPerCta;
+  ovf_warp_kernel<E><<<ctas, kOvfWarpsPerCta * 32, per_warp * kOvfWarpsPerCta, stream>>>(p, n_groups);
+}
+
 int launch_ovf(int n_groups, int n, int k, const float* scores, int32_t* keep_idx,
                int32_t* src_rows, float* sel_var, float* kept_scores, float* adv, float adv_eps,
                const int32_t* traj_in, int32_t* traj_out, int32_t* status, cudaStream_t stream) {
@@ -261,8 +470,14 @@ int launch_ovf(int n_groups, int n, int k, const float* scores, int32_t* keep_id
   p.n = n;
   p.k = k;
   p.adv_eps = adv_eps;
-  const size_t smem = (size_t)n * 8 + (size_t)(k + 1) * 4 * 8 + (size_t)n * 4;
-  ovf_select_kernel<<<n_groups, kOvfThreads, smem, stream>>>(p);
+  if (n <= 32)       launch_ovf_warp<1>(p, n_groups, stream);
+  else if (n <= 64)  launch_ovf_warp<2>(p, n_groups, stream);
+  else if (n <= 128) launch_ovf_warp<4>(p, n_groups, stream);
+  else if (n <= 256) launch_ovf_warp<8>(p, n_groups, stream);
+  else {
+    const size_t smem = (size_t)n * 8 + (size_t)(k + 1) * 4 * 8 + (size_t)n * 4;
+    ovf_select_kernel<<<n_groups, kOvfThreads, smem, stream>>>(p);
+  }
   PG_LAUNCH_CHECK();
   return PG_OK;
 }
