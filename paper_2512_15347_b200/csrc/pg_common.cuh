@@ -76,7 +76,9 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
 __device__ __forceinline__ float normal_pair(uint32_t r0, uint32_t r1, float& a, float& b) {
   const float k1 = (float)(r0 >> 8);
   const float u1 = fmaf(k1, 5.9604644775390625e-8f, 5.9604644775390625e-8f);
-  float neg2ln = -1.3862943611198906f * __log2f(u1);           // -2 ln(u1) = -2 ln2 * log2(u1)
+  float lg;                                                     // u1 >= 2^-24: never subnormal
+  asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(u1));
+  float neg2ln = -1.3862943611198906f * lg;                     // -2 ln(u1) = -2 ln2 * log2(u1)
   const float w = 1.0f - u1;                                     // exact (Sterbenz / 24-bit grid)
   // -2 ln(1 - w) = 2w + w^2 + (2/3) w^3 + (1/2) w^4 + ...
   float ser = fmaf(w, 0.5f, 0.66666666666666667f);
@@ -87,8 +89,10 @@ __device__ __forceinline__ float normal_pair(uint32_t r0, uint32_t r1, float& a,
   float radius;
   asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(radius) : "f"(neg2ln));
   const float turn = fmaf((float)(r1 >> 8), 5.9604644775390625e-8f, -0.5f);  // u2 - 1/2, exact
+  const float angle = 6.283185307179586f * turn;
   float s, c;
-  __sincosf(6.283185307179586f * turn, &s, &c);
+  asm("sin.approx.ftz.f32 %0, %1;" : "=f"(s) : "f"(angle));
+  asm("cos.approx.ftz.f32 %0, %1;" : "=f"(c) : "f"(angle));
   a = -radius * c;
   b = -radius * s;
   return neg2ln;
@@ -113,8 +117,14 @@ __device__ __forceinline__ double warp_sum(double v) {
 constexpr int kRowThreads = 256;
 constexpr int kRowWarps = kRowThreads / 32;
 constexpr int kMinChunkQuads = kRowThreads * 2;        // 512 quads  = 2048 elements
-constexpr int kMaxChunkQuads = kMinChunkQuads * 16;    // 8192 quads = 32768 elements
-constexpr long long kWantedCtas = 148LL * 4 * 16;      // enough CTAs for ~16 waves on 148 SMs
+#ifndef PG_MAX_CHUNK_MULT
+#define PG_MAX_CHUNK_MULT 16
+#endif
+constexpr int kMaxChunkQuads = kMinChunkQuads * PG_MAX_CHUNK_MULT;    // 8192 quads = 32768 elements
+#ifndef PG_WANTED_WAVES
+#define PG_WANTED_WAVES 16
+#endif
+constexpr long long kWantedCtas = 148LL * 4 * PG_WANTED_WAVES;   // CTAs for that many waves on 148 SMs
 
 struct RowGeometry {
   int chunk_quads;   // quads per CTA

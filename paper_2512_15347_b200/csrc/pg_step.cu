@@ -52,9 +52,46 @@ template <typename T> struct VelReg;
 template <> struct VelReg<float> { using type = VelF32; };
 template <> struct VelReg<__nv_bfloat16> { using type = VelBf16; };
 
+#ifndef PG_STEP_UNROLL
+#define PG_STEP_UNROLL 2       // quads per thread and loop iteration (the next batch is in flight)
+#endif
+#ifndef PG_STEP_MIN_CTAS
+#define PG_STEP_MIN_CTAS 5     // __launch_bounds__ minimum resident CTAs per SM
+#endif
+constexpr int kStepUnroll = PG_STEP_UNROLL;
+
+// One quad: mean of the transition, noise, store, radius-term accumulation.
+template <bool kNoise, bool kUnitCx>
+__device__ __forceinline__ void step_quad(const StepParams& p, uint32_t traj, int q, const float4& xv,
+                                          const float4& vv, float4* __restrict__ xout, float& acc) {
+  float4 m;
+  if (kUnitCx) {
+    m.x = fmaf(p.c_v, vv.x, xv.x);
+    m.y = fmaf(p.c_v, vv.y, xv.y);
+    m.z = fmaf(p.c_v, vv.z, xv.z);
+    m.w = fmaf(p.c_v, vv.w, xv.w);
+  } else {
+    m.x = fmaf(p.c_v, vv.x, p.c_x * xv.x);
+    m.y = fmaf(p.c_v, vv.y, p.c_x * xv.y);
+    m.z = fmaf(p.c_v, vv.z, p.c_x * xv.z);
+    m.w = fmaf(p.c_v, vv.w, p.c_x * xv.w);
+  }
+  if (kNoise) {
+    const uint4 r = philox4x32_10((uint32_t)q, p.step, traj, 0u, p.rk);
+    float n0, n1, n2, n3;
+    acc += normal_pair(r.x, r.y, n0, n1);
+    acc += normal_pair(r.z, r.w, n2, n3);
+    m.x = fmaf(p.noise_std, n0, m.x);
+    m.y = fmaf(p.noise_std, n1, m.y);
+    m.z = fmaf(p.noise_std, n2, m.z);
+    m.w = fmaf(p.noise_std, n3, m.w);
+  }
+  __stcs(xout + q, m);
+}
+
 // kNoise: noise_std > 0.  kUnitCx: c_x == 1 (drift = prediction), one FMA per element less.
 template <typename VelT, bool kNoise, bool kUnitCx>
-__global__ void __launch_bounds__(kRowThreads)
+__global__ void __launch_bounds__(kRowThreads, PG_STEP_MIN_CTAS)
 step_kernel(const __grid_constant__ StepParams p) {
   using VReg = typename VelReg<VelT>::type;
   const int row = blockIdx.x / p.chunks;
@@ -62,54 +99,35 @@ step_kernel(const __grid_constant__ StepParams p) {
   const int src = p.src_rows ? p.src_rows[row] : row;
   const uint32_t traj = (uint32_t)p.traj_id[row];
 
-  const float4* xin = reinterpret_cast<const float4*>(p.x_in) + (size_t)src * p.quads_per_row;
-  const VelT* vel = reinterpret_cast<const VelT*>(p.vel) + (size_t)src * p.quads_per_row * 4;
-  float4* xout = reinterpret_cast<float4*>(p.x_out) + (size_t)row * p.quads_per_row;
+  const float4* __restrict__ xin = reinterpret_cast<const float4*>(p.x_in) + (size_t)src * p.quads_per_row;
+  const VelT* __restrict__ vel = reinterpret_cast<const VelT*>(p.vel) + (size_t)src * p.quads_per_row * 4;
+  float4* __restrict__ xout = reinterpret_cast<float4*>(p.x_out) + (size_t)row * p.quads_per_row;
   const int q_begin = chunk * p.chunk_quads;
   const int q_end = min(q_begin + p.chunk_quads, p.quads_per_row);
 
   float acc = 0.f;
-  auto process = [&](int q, const float4& xv, const VReg& vraw) {
-    const float4 vv = vel_f32(vraw);
-    float4 m;
-    if (kUnitCx) {
-      m.x = fmaf(p.c_v, vv.x, xv.x);
-      m.y = fmaf(p.c_v, vv.y, xv.y);
-      m.z = fmaf(p.c_v, vv.z, xv.z);
-      m.w = fmaf(p.c_v, vv.w, xv.w);
-    } else {
-      m.x = fmaf(p.c_v, vv.x, p.c_x * xv.x);
-      m.y = fmaf(p.c_v, vv.y, p.c_x * xv.y);
-      m.z = fmaf(p.c_v, vv.z, p.c_x * xv.z);
-      m.w = fmaf(p.c_v, vv.w, p.c_x * xv.w);
-    }
-    if (kNoise) {
-      const uint4 r = philox4x32_10((uint32_t)q, p.step, traj, 0u, p.rk);
-      float n0, n1, n2, n3;
-      acc += normal_pair(r.x, r.y, n0, n1);
-      acc += normal_pair(r.z, r.w, n2, n3);
-      m.x = fmaf(p.noise_std, n0, m.x);
-      m.y = fmaf(p.noise_std, n1, m.y);
-      m.z = fmaf(p.noise_std, n2, m.z);
-      m.w = fmaf(p.noise_std, n3, m.w);
-    }
-    __stcs(xout + q, m);
-  };
-
+  float4 xv[kStepUnroll], nx[kStepUnroll];
+  VReg vv[kStepUnroll], nv[kStepUnroll];
   int q = q_begin + threadIdx.x;
-  float4 xa, xb;
-  VReg va, vb;
-  if (q < q_end) { xa = __ldcs(xin + q); load_vel(vel, (size_t)q, va); }
-  if (q + kRowThreads < q_end) { xb = __ldcs(xin + q + kRowThreads); load_vel(vel, (size_t)q + kRowThreads, vb); }
+#pragma unroll
+  for (int u = 0; u < kStepUnroll; ++u) {
+    const int qq = q + u * kRowThreads;
+    if (qq < q_end) { xv[u] = __ldcs(xin + qq); load_vel(vel, (size_t)qq, vv[u]); }
+  }
   while (q < q_end) {
-    const int nq = q + 2 * kRowThreads;
-    float4 nxa, nxb;
-    VReg nva, nvb;
-    if (nq < q_end) { nxa = __ldcs(xin + nq); load_vel(vel, (size_t)nq, nva); }
-    if (nq + kRowThreads < q_end) { nxb = __ldcs(xin + nq + kRowThreads); load_vel(vel, (size_t)nq + kRowThreads, nvb); }
-    process(q, xa, va);
-    if (q + kRowThreads < q_end) process(q + kRowThreads, xb, vb);
-    xa = nxa; xb = nxb; va = nva; vb = nvb;
+    const int nq = q + kStepUnroll * kRowThreads;
+#pragma unroll
+    for (int u = 0; u < kStepUnroll; ++u) {
+      const int qq = nq + u * kRowThreads;
+      if (qq < q_end) { nx[u] = __ldcs(xin + qq); load_vel(vel, (size_t)qq, nv[u]); }
+    }
+#pragma unroll
+    for (int u = 0; u < kStepUnroll; ++u) {
+      const int qq = q + u * kRowThreads;
+      if (qq < q_end) step_quad<kNoise, kUnitCx>(p, traj, qq, xv[u], vel_f32(vv[u]), xout, acc);
+    }
+#pragma unroll
+    for (int u = 0; u < kStepUnroll; ++u) { xv[u] = nx[u]; vv[u] = nv[u]; }
     q = nq;
   }
 
@@ -119,10 +137,10 @@ step_kernel(const __grid_constant__ StepParams p) {
   }
   acc = warp_sum(acc);
   const int slots = p.chunks * kRowWarps;
+  float* logp_out = p.logp_out;
+  const double logp_const = p.logp_const, logp_scale = p.logp_scale;
   finish_row(acc, row, chunk * kRowWarps + (threadIdx.x >> 5), slots, p.partials, p.tickets,
-             [&](double sum) {
-               p.logp_out[row] = (float)((-0.5 * sum - p.logp_const) * p.logp_scale);
-             });
+             [=](double sum) { logp_out[row] = (float)((-0.5 * sum - logp_const) * logp_scale); });
 }
 
 template <typename VelT>
