@@ -230,14 +230,14 @@ int pg_rollout_host(const pg_config *cfg, const pg_step_coef *step_coef,
  * start-up, code in a latency-critical section where cudaMalloc (which may synchronise the
  * device) is unwelcome.  pg_score needs a handle and pg_rollout_init allocates; this call
  * needs neither.  Its reduction scratch is a fixed array inside the library image
- * (about 1 MB, resident on every GPU that loads the library until the process exits).
+ * (about 300 KB, resident on every GPU that loads the library until the process exits).
  *
  *   scores_out[i] = mean_e(p_x * x[i][e] + p_v * vel[i][e]),  i < n_rows
  *   x [n_rows, elems] fp32, vel [n_rows, elems] fp32 or bf16 per vel_dtype (not read and may
  *   be NULL when p_v == 0), scores_out [n_rows] fp32: caller-owned device memory, x and vel
  *   16-byte aligned.  elems a positive multiple of 4.
  *
- * Limits: n_rows <= PG_STATIC_MAX_ROWS and 8 * n_rows * ceil(elems / 32768) <=
+ * Limits: n_rows <= PG_STATIC_MAX_ROWS and n_rows * ceil(elems / 32768) <=
  * PG_STATIC_MAX_PARTIALS; beyond either the call returns PG_ECAPACITY and does nothing
  * (split the rows over several calls).  Calls no cudaMalloc / cudaFree.  The first call on
  * each device looks up the device address of the built-in array; make that first call
@@ -247,7 +247,7 @@ int pg_rollout_host(const pg_config *cfg, const pg_step_coef *step_coef,
  * on one stream or order them with events.
  */
 #define PG_STATIC_MAX_ROWS     8192
-#define PG_STATIC_MAX_PARTIALS 262144
+#define PG_STATIC_MAX_PARTIALS 65536
 int pg_score_static(int32_t n_rows, int32_t elems, int32_t vel_dtype, const pg_preview_coef *coef,
                     const float *x, const void *vel, float *scores_out, void *stream);
 

@@ -15,7 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libprogrpo.so")
 
 OK, EINVAL, ESTATE, ECUDA, ENONFINITE, ETIMEOUT, ENOMEM, ECAPACITY = 0, -1, -2, -3, -4, -5, -6, -7
-STATIC_MAX_ROWS, STATIC_MAX_PARTIALS = 8192, 262144
+STATIC_MAX_ROWS, STATIC_MAX_PARTIALS = 8192, 65536
 VEL_F32, VEL_BF16 = 0, 1
 MAX_GROUP = 1024
 

@@ -112,27 +112,21 @@ __device__ __forceinline__ double warp_sum(double v) {
 
 // ---------------------------------------------------------------- launch geometry
 // Row-streaming kernels (step, score): a CTA of kRowThreads threads handles one chunk of one
-// row; a chunk is chunk_quads 4-element quads, a multiple of kRowThreads * 2.  Every warp of
-// every CTA contributes one partial sum, so a row owns chunks * kRowWarps partial slots.
+// row and contributes one partial sum, so a row owns `chunks` partial slots.  Chunks are
+// 2048..8192 quads (4-element groups): short chunks pay the end-of-CTA reduction (a barrier, a
+// fence and an atomic) too often, long ones leave too few CTAs to fill 148 SMs evenly.
 constexpr int kRowThreads = 256;
 constexpr int kRowWarps = kRowThreads / 32;
-constexpr int kMinChunkQuads = kRowThreads * 2;        // 512 quads  = 2048 elements
-#ifndef PG_MAX_CHUNK_MULT
-#define PG_MAX_CHUNK_MULT 16
-#endif
-constexpr int kMaxChunkQuads = kMinChunkQuads * PG_MAX_CHUNK_MULT;    // 8192 quads = 32768 elements
-#ifndef PG_WANTED_WAVES
-#define PG_WANTED_WAVES 16
-#endif
-constexpr long long kWantedCtas = 148LL * 4 * PG_WANTED_WAVES;   // CTAs for that many waves on 148 SMs
+constexpr int kMinChunkQuads = 2048;                   // 8192 elements
+constexpr int kMaxChunkQuads = 8192;                   // 32768 elements
+constexpr long long kWantedCtas = 148LL * 4 * 16;      // CTAs for ~16 waves at 4 CTAs per SM
 
 struct RowGeometry {
   int chunk_quads;   // quads per CTA
-  int chunks;        // CTAs per row
-  int slots;         // partial sums per row = chunks * kRowWarps
+  int chunks;        // CTAs per row = partial sums per row
 };
 
-// Longest chunk (fewest CTA start-ups and reductions) that still leaves kWantedCtas CTAs.
+// Longest chunk that still leaves kWantedCtas CTAs, but never shorter than kMinChunkQuads.
 inline RowGeometry row_geometry(long long rows, int elems, int forced_chunk_quads = 0) {
   const int quads = elems / 4;
   int cq = kMaxChunkQuads;
@@ -144,32 +138,42 @@ inline RowGeometry row_geometry(long long rows, int elems, int forced_chunk_quad
   RowGeometry g;
   g.chunk_quads = cq;
   g.chunks = (quads + cq - 1) / cq;
-  g.slots = g.chunks * kRowWarps;
   return g;
 }
 
 #ifdef __CUDACC__
-// Per-row reduction without any CTA barrier or waiting.  Every warp of every CTA of the row
-// calls this once with its total (all lanes hold it).  The warp stores its total in its fixed
-// slot and takes a ticket; the warp that draws the last ticket adds all slots in slot order
-// (fp64) and hands the sum to fin(sum) on lane 0.  The result is independent of the order in
-// which warps arrive.  tickets[row] is left at zero for the next launch.
+// Per-row reduction in a fixed shape, without waiting on other CTAs.  Every thread of every CTA
+// of the row calls this once with its warp's total (all lanes hold it).  Warp totals are
+// combined through shared memory in warp order; warp 0 stores the CTA total in the CTA's fixed
+// slot and takes a ticket; the CTA that draws the last ticket adds all slots in slot order
+// (fp64) and hands the sum to fin(sum) on thread 0.  The result is independent of the order in
+// which CTAs run.  tickets[row] is left at zero for the next launch.
 template <typename Fin>
-__device__ __forceinline__ void finish_row(float warp_total, int row, int slot, int slots,
+__device__ __forceinline__ void finish_row(float warp_total, int row, int chunk, int chunks,
                                            float* partials, unsigned int* tickets, Fin fin) {
+  __shared__ float warp_part[kRowWarps];
   const int lane = threadIdx.x & 31;
+  if (lane == 0) warp_part[threadIdx.x >> 5] = warp_total;
+  __syncthreads();
+  if (threadIdx.x >= 32) return;
+  float v = lane < kRowWarps ? warp_part[lane] : 0.f;
+  v = warp_sum(v);
+  if (chunks == 1) {
+    if (lane == 0) fin((double)v);
+    return;
+  }
   int last = 0;
   if (lane == 0) {
-    partials[(size_t)row * slots + slot] = warp_total;
+    partials[(size_t)row * chunks + chunk] = v;
     __threadfence();
     const unsigned int t = atomicAdd(&tickets[row], 1u);
-    last = (t == (unsigned int)slots - 1u);
+    last = (t == (unsigned int)chunks - 1u);
   }
   last = __shfl_sync(0xFFFFFFFFu, last, 0);
   if (!last) return;
   __threadfence();
   double s = 0.0;
-  for (int c = lane; c < slots; c += 32) s += (double)__ldcg(&partials[(size_t)row * slots + c]);
+  for (int c = lane; c < chunks; c += 32) s += (double)__ldcg(&partials[(size_t)row * chunks + c]);
   s = warp_sum(s);
   if (lane == 0) {
     fin(s);
@@ -180,7 +184,7 @@ __device__ __forceinline__ void finish_row(float warp_total, int row, int slot, 
 
 // ---------------------------------------------------------------- launchers (device pointers)
 struct RowScratch {
-  float* partials;        // [rows * row_geometry(rows, elems).slots]
+  float* partials;        // [rows * row_geometry(rows, elems).chunks]
   unsigned int* tickets;  // [rows], zero between launches
 };
 

@@ -81,10 +81,10 @@ int pg_rollout_init(const pg_config* cfg, pg_rollout** out) {
   h->k_cur = cfg->n_expand;
   const size_t rows = (size_t)cfg->n_groups * cfg->n_expand;
   // partial-sum slots: the largest need over the row counts this schedule will launch with
-  size_t slots = rows * (size_t)pg::row_geometry((long long)rows, cfg->elems).slots;
+  size_t slots = rows * (size_t)pg::row_geometry((long long)rows, cfg->elems).chunks;
   for (int i = 0; i < cfg->n_stages; ++i) {
     const long long r = (long long)cfg->n_groups * cfg->stage_keep[i];
-    const size_t need = (size_t)r * (size_t)pg::row_geometry(r, cfg->elems).slots;
+    const size_t need = (size_t)r * (size_t)pg::row_geometry(r, cfg->elems).chunks;
     if (need > slots) slots = need;
   }
   cudaError_t e = cudaGetDevice(&h->device);

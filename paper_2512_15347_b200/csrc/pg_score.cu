@@ -91,8 +91,7 @@ score_kernel(const __grid_constant__ ScoreParams p) {
   }
 
   acc = warp_sum(acc);
-  const int slots = p.chunks * kRowWarps;
-  finish_row(acc, row, chunk * kRowWarps + (threadIdx.x >> 5), slots, p.partials, p.tickets,
+  finish_row(acc, row, chunk, p.chunks, p.partials, p.tickets,
              [&](double sum) { p.scores_out[row] = (float)(sum * p.inv_d); });
 }
 

@@ -7,7 +7,7 @@
 // handle, and creating a handle allocates its reduction scratch.  This entry point needs no
 // handle: the reduction scratch (per-row partial sums and the per-row arrival counters) lives in
 // a fixed array that is part of the library image, so every GPU that loads the library carries
-// it (about 1 MB) until the process exits.
+// it (about 300 KB) until the process exits.
 //
 // The first call on a device looks up the device address of that array; host code cannot use
 // the array's name as a pointer (on the host the name denotes a stand-in object, not device
@@ -62,7 +62,7 @@ extern "C" int pg_score_static(int32_t n_rows, int32_t elems, int32_t vel_dtype,
   // capacity of the built-in scratch: PG_STATIC_MAX_ROWS rows, PG_STATIC_MAX_PARTIALS partial sums
   if (n_rows > kStaticMaxRows) return PG_ECAPACITY;
   const pg::RowGeometry geo = pg::row_geometry(n_rows, elems, pg::kMaxChunkQuads);
-  const size_t need = (size_t)n_rows * (size_t)geo.slots;
+  const size_t need = (size_t)n_rows * (size_t)geo.chunks;
   if (need > kStaticMaxPartials) return PG_ECAPACITY;
 
   StaticScratch* s = nullptr;

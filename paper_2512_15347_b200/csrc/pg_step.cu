@@ -136,10 +136,9 @@ step_kernel(const __grid_constant__ StepParams p) {
     return;
   }
   acc = warp_sum(acc);
-  const int slots = p.chunks * kRowWarps;
   float* logp_out = p.logp_out;
   const double logp_const = p.logp_const, logp_scale = p.logp_scale;
-  finish_row(acc, row, chunk * kRowWarps + (threadIdx.x >> 5), slots, p.partials, p.tickets,
+  finish_row(acc, row, chunk, p.chunks, p.partials, p.tickets,
              [=](double sum) { logp_out[row] = (float)((-0.5 * sum - logp_const) * logp_scale); });
 }
 

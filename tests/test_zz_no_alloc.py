@@ -50,7 +50,7 @@ def test_static_score_refuses_what_does_not_fit():
         B.score_static(B.STATIC_MAX_ROWS + 1, 64, B.VEL_F32, (1.0, 0.0), x, None, out)
     assert e.value.code == B.ECAPACITY
     with pytest.raises(B.PgError) as e:       # rows fit, rows x chunks does not
-        B.score_static(B.STATIC_MAX_ROWS, 32768 * 4 + 4, B.VEL_F32, (1.0, 0.0), x, None, out)
+        B.score_static(B.STATIC_MAX_ROWS, 32768 * 8 + 4, B.VEL_F32, (1.0, 0.0), x, None, out)
     assert e.value.code == B.ECAPACITY
     with pytest.raises(B.PgError) as e:
         B.score_static(8, 66, B.VEL_F32, (1.0, 0.0), x, None, out)
