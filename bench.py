@@ -28,6 +28,12 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) over algorithmic bytes of the step
+# kernel, from the ncu capture summarised in profiles/step_kernel_bf16_1024rows.txt (1024-row
+# launch: 2.642 GB measured, 2.684 GB algorithmic).  Set to None whenever the kernel changes
+# until the counters are taken again.
+STEP_KERNEL_TRAFFIC_RATIO = 0.984
+
 METRIC = "latent-steps/s (SDE step+logprob+OVF prune)"
 UNIT = "latent-steps/s"
 
@@ -304,7 +310,12 @@ def run_ours(args):
                 "roofline": {"bound": "hbm", "kernel": "step_kernel<bf16> (SDE step + log-prob)",
                              "achieved": step_gbs, "peak": peak, "unit": "GB/s",
                              "frac": step_gbs / peak, "peak_kind": peak_kind,
-                             "frac_of_8TBs_nominal": step_gbs / 8000.0, "traffic": None,
+                             "frac_of_8TBs_nominal": step_gbs / 8000.0,
+                             "bytes_per_launch": step_bytes / kinds["step"]["launches"],
+                             "traffic": (None if STEP_KERNEL_TRAFFIC_RATIO is None else
+                                         STEP_KERNEL_TRAFFIC_RATIO * step_bytes / kinds["step"]["launches"]),
+                             "traffic_source": "ncu capture of the 1024-row launch, scaled by rows "
+                                               "(traffic is proportional to rows x elements)",
                              "bytes_per_element_step": 8 + vel_bytes},
                 "kernels": {k: {"ms_per_rollout": v["ms"] / args.steps, "launches_per_rollout":
                                 v["launches"] // args.steps} for k, v in kinds.items()},
