@@ -178,6 +178,7 @@ def run_ours(args):
     import torch
     from paper_2512_15347_b200 import binding as B
     from paper_2512_15347_b200 import workloads as wl
+    from paper_2512_15347_b200 import sharding
     from paper_2512_15347_b200.rollout import Rollout
 
     rank = int(os.environ.get("RANK", "0"))
@@ -199,7 +200,7 @@ def run_ours(args):
 
     torch.cuda.set_device(local)
     dist = None
-    if world > 1:
+    if world > 1 or "TORCHELASTIC_RUN_ID" in os.environ:      # launched by torch.distributed.run
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     B.lib()
@@ -209,7 +210,7 @@ def run_ours(args):
 
     dt = torch.bfloat16 if w.vel_dtype == "bf16" else torch.float32
     ro = Rollout(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, dt, adv_eps=w.adv_eps,
-                 group_offset=rank * w.n_groups)
+                 group_offset=sharding.weak_shard(w.n_groups, rank)[0])
     x0 = wl.initial_latents(wr, device=dev)
     vels = [wl.normal_velocity(wr, s, w.n_groups * w.rows_before(s), device=dev)
             for s in range(w.n_steps)]
@@ -245,9 +246,7 @@ def run_ours(args):
     total_ms = ev0.elapsed_time(ev1)
     if dist is not None:
         dist.barrier()
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+        total_ms = sharding.max_over_ranks(total_ms, dist, dev)
 
     # per-kernel device times from the events recorded inside the timed region
     kinds = {}
@@ -333,7 +332,7 @@ def run_e2e(B, wl, w, wr, rank, dist, dev, args):
     import torch
     cfg = B.make_config(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed,
                         B.VEL_BF16 if w.vel_dtype == "bf16" else B.VEL_F32, adv_eps=w.adv_eps,
-                        group_offset=rank * w.n_groups)
+                        group_offset=rank * w.n_groups)  # = sharding.weak_shard(...)[0]
     ws = torch.empty(B.rollout_host_workspace_bytes(cfg), dtype=torch.uint8, device=dev)
     dt = torch.bfloat16 if w.vel_dtype == "bf16" else torch.float32
     # host inputs: pinned; filled from a seeded CPU generator block by block (content does not
@@ -374,11 +373,8 @@ def run_e2e(B, wl, w, wr, rank, dist, dev, args):
         call()
     b.record()
     torch.cuda.synchronize()
-    ms = a.elapsed_time(b)
-    if dist is not None:
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    from paper_2512_15347_b200 import sharding
+    ms = sharding.max_over_ranks(a.elapsed_time(b), dist, dev)
     world = 1 if dist is None else dist.get_world_size()
     h2d = x0.numel() * 4 + sum(v.numel() * v.element_size() for v in vels)
     d2h = x_final.numel() * 4 + logp.numel() * 4 + keep.numel() * 4 + adv.numel() * 4 + ids.numel() * 4
