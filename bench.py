@@ -166,7 +166,9 @@ def _config(w, args):
                         + f" at steps {[s for s, _ in w.stages]} of {w.n_steps}, d={w.elems}, "
                         f"fp32 latents, {w.vel_dtype} predictions, seed {w.seed}",
             "groups_per_gpu": w.n_groups, "latent_steps_per_rollout": w.traj_steps,
-            "l2": "inputs larger than L2: no flush (state %.2f GB, predictions %.2f GB per rollout)"
+            "l2": ("inputs larger than L2: no flush" if w.n_groups * w.n_expand * w.elems * 4 > 256e6
+                   else "state fits L2 (L2-assisted numbers, launch-bound workload)")
+                  + " (state %.3f GB, predictions %.3f GB per rollout)"
                   % (w.n_groups * w.n_expand * w.elems * 4 / 1e9,
                      w.element_steps * (2 if w.vel_dtype == "bf16" else 4) / 1e9),
             "parallelism": f"groups sharded over {args.gpus} GPU(s), no collective"}
@@ -212,12 +214,32 @@ def run_ours(args):
     ro = Rollout(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, dt, adv_eps=w.adv_eps,
                  group_offset=sharding.weak_shard(w.n_groups, rank)[0])
     x0 = wl.initial_latents(wr, device=dev)
-    vels = [wl.normal_velocity(wr, s, w.n_groups * w.rows_before(s), device=dev)
-            for s in range(w.n_steps)]
+    ext = fin = None
+    if w.velocity == "affine":
+        a_c, b_c = wl.affine_field(wr, device=dev)
+        velocity = lambda s, x: wl.affine_velocity(x, a_c, b_c)   # stand-in network, inside the timing
+    else:
+        vels = [wl.normal_velocity(wr, s, w.n_groups * w.rows_before(s), device=dev)
+                for s in range(w.n_steps)]
+        velocity = lambda s, x: vels[s]
+    if w.scores == "external":
+        # stand-in reward model: one score table per stage, looked up by original trajectory
+        tables = [torch.from_numpy(wl.clustered_scores(w.n_groups, w.n_expand, wr.seed, st, cluster_sigma=0.05,
+                                                       outlier_frac=0.15, outlier_scale=0.3, nu=3.0)
+                                   ).reshape(-1).to(dev) for st in list(range(len(w.stages))) + [99]]
+        base = sharding.weak_shard(w.n_groups, rank)[0] * w.n_expand
+
+        def lookup(table):
+            ids = torch.empty(ro.n_active, device=dev, dtype=torch.int32)
+            B.rollout_traj_ids(ro.h, ids)
+            return table[(ids - base).long()]
+        ext = lambda stage: lookup(tables[stage])
+        fin = lambda: lookup(tables[-1])
     torch.cuda.synchronize()
 
     def one_rollout(trace=None):
-        return ro.run(x0, w.step_coef, w.preview_coef, lambda s, x: vels[s], trace=trace)
+        return ro.run(x0, w.step_coef, w.preview_coef, velocity, external_scores=ext,
+                      final_rewards=fin, trace=trace)
 
     for _ in range(max(args.warmup, 3)):
         one_rollout()
@@ -389,7 +411,7 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="large", choices=["large", "sd15", "tiny"])
+    ap.add_argument("--workload", default="large", choices=["large", "sd3", "sd15", "tiny"])
     ap.add_argument("--groups", type=int, default=0,
                     help="prompt groups per GPU (default: the workload's own; smaller for profiling)")
     ap.add_argument("--no-e2e", action="store_true")
