@@ -218,7 +218,9 @@ int pg_ovf_select_batched(int32_t n_groups, int32_t n, int32_t k, const float* s
                           int32_t* keep_idx, float* kept_scores, float* adv, float adv_eps,
                           int32_t* status, void* stream) {
   if (n_groups < 0 || n < 1 || n > PG_MAX_GROUP || k < 1 || k > n) return PG_EINVAL;
-  if (!scores || !keep_idx || !(adv_eps >= 0.f)) return PG_EINVAL;
+  if (!(adv_eps >= 0.f)) return PG_EINVAL;
+  if (n_groups == 0) return PG_OK;
+  if (!scores || !keep_idx) return PG_EINVAL;
   return pg::launch_ovf(n_groups, n, k, scores, keep_idx, nullptr, nullptr, kept_scores, adv,
                         adv_eps, nullptr, nullptr, status, (cudaStream_t)stream);
 }
