@@ -299,3 +299,68 @@ def rollout(x0: np.ndarray, n_groups: int, n_expand: int, n_steps: int,
     res.rewards = rw
     res.adv, res.mean, res.std = advantages(rw, adv_eps)
     return res
+
+
+# ---------------------------------------------------------------- policy update (Eq. ratio_method, Eq. pro_grpo_method)
+
+def policy_logprob(x: np.ndarray, x_next: np.ndarray, vel: np.ndarray, vel_ref: Optional[np.ndarray],
+                   c_x: float, c_v: float, noise_std: float, logp_mean: bool = False):
+    """log pi_theta of the stored transitions under a new prediction, and KL to a reference."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    x_next = np.ascontiguousarray(x_next, dtype=np.float32)
+    vel, vdt = _vel_arg(vel)
+    n, d = x.shape
+    logp = np.empty(n, dtype=np.float64)
+    kl = None
+    if vel_ref is not None:
+        vel_ref, vdt2 = _vel_arg(vel_ref)
+        assert vdt2 == vdt
+        kl = np.empty(n, dtype=np.float64)
+    rc = _load().og_policy_logprob(ctypes.c_int64(n), ctypes.c_int64(d), _ptr(x), _ptr(x_next), _ptr(vel),
+                                   _ptr(vel_ref), ctypes.c_int(vdt), ctypes.c_double(c_x),
+                                   ctypes.c_double(c_v), ctypes.c_double(noise_std),
+                                   ctypes.c_int(1 if logp_mean else 0), _ptr(logp), _ptr(kl))
+    _check(rc, "policy_logprob")
+    return logp, kl
+
+
+def policy_objective(logp_new: np.ndarray, logp_old: np.ndarray, kl: Optional[np.ndarray],
+                     adv: np.ndarray, clip_eps: float, beta: float):
+    """Clipped surrogate objective, ratios and dJ/dlogp_new for [T, n] log-probs."""
+    logp_new = np.ascontiguousarray(logp_new, dtype=np.float64)
+    logp_old = np.ascontiguousarray(logp_old, dtype=np.float64)
+    adv = np.ascontiguousarray(adv, dtype=np.float64)
+    T, n = logp_new.shape
+    assert logp_old.shape == (T, n) and adv.shape == (n,)
+    if kl is not None:
+        kl = np.ascontiguousarray(kl, dtype=np.float64)
+        assert kl.shape == (T, n)
+    ratio = np.empty((T, n), dtype=np.float64)
+    dlogp = np.empty((T, n), dtype=np.float64)
+    obj = ctypes.c_double(0.0)
+    rc = _load().og_policy_objective(ctypes.c_int64(T), ctypes.c_int64(n), _ptr(logp_new), _ptr(logp_old),
+                                     _ptr(kl), _ptr(adv), ctypes.c_double(clip_eps), ctypes.c_double(beta),
+                                     _ptr(ratio), _ptr(dlogp), ctypes.byref(obj))
+    _check(rc, "policy_objective")
+    return float(obj.value), ratio, dlogp
+
+
+def policy_backward(x: np.ndarray, x_next: np.ndarray, vel: np.ndarray, vel_ref: Optional[np.ndarray],
+                    c_x: float, c_v: float, noise_std: float, dlogp: np.ndarray, dkl: float,
+                    logp_mean: bool = False) -> np.ndarray:
+    """dJ/dvel for one step (fp64 [n, d])."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    x_next = np.ascontiguousarray(x_next, dtype=np.float32)
+    vel, vdt = _vel_arg(vel)
+    if vel_ref is not None:
+        vel_ref, _ = _vel_arg(vel_ref)
+    dlogp = np.ascontiguousarray(dlogp, dtype=np.float64)
+    n, d = x.shape
+    grad = np.empty((n, d), dtype=np.float64)
+    rc = _load().og_policy_backward(ctypes.c_int64(n), ctypes.c_int64(d), _ptr(x), _ptr(x_next), _ptr(vel),
+                                    _ptr(vel_ref), ctypes.c_int(vdt), ctypes.c_double(c_x),
+                                    ctypes.c_double(c_v), ctypes.c_double(noise_std),
+                                    ctypes.c_int(1 if logp_mean else 0), _ptr(dlogp), ctypes.c_double(dkl),
+                                    _ptr(grad))
+    _check(rc, "policy_backward")
+    return grad

@@ -17,7 +17,9 @@
  * Parity pins (tests/test_oracle_*.py): Philox known answers, normal-sample
  * statistics, Gaussian log-density against scipy, moment recursions of the
  * Euler-Maruyama step, exhaustive subset search for OVF, numpy statistics
- * for the advantages.  No function in this file is "parity unpinned".
+ * for the advantages; for the policy update scipy densities, a numerically
+ * integrated KL, hand-worked clipping cases and finite differences.  No
+ * function in this file is "parity unpinned".
  */
 #include <math.h>
 #include <stdint.h>
@@ -473,4 +475,112 @@ int og_num_threads(void)
 #else
     return 1;
 #endif
+}
+
+/* ------------------------------------------------------------------ */
+/* Policy update on the survivors (Section 5.1, Eq. "ratio_method",    */
+/* Eq. "pro_grpo_method"; GRPO loss of Section 3.3)                    */
+/* ------------------------------------------------------------------ */
+
+/*
+ * Log-density of the stored transition x -> x_next under the Gaussian policy
+ * that a (new) prediction `vel` induces, and the KL divergence from the policy
+ * of a reference prediction `vel_ref`:
+ *     m      = c_x x + c_v vel ,   m_ref = c_x x + c_v vel_ref
+ *     log pi = -1/2 sum ((x_next - m)/s)^2 - d/2 ln(2 pi s^2)        (/ d if logp_mean)
+ *     KL( N(m, s^2 I) || N(m_ref, s^2 I) ) = sum (m - m_ref)^2 / (2 s^2)   (/ d if logp_mean)
+ * (two Gaussians with the same covariance: only the mean shift contributes).
+ * vel_ref and kl_out may be NULL together.
+ */
+int og_policy_logprob(int64_t n, int64_t d, const float *x, const float *x_next,
+                      const void *vel, const void *vel_ref, int vel_dtype,
+                      double c_x, double c_v, double noise_std, int logp_mean,
+                      double *logp_out, double *kl_out)
+{
+    if (n < 0 || d <= 0 || !x || !x_next || !vel || !logp_out || !(noise_std > 0.0)) return OG_EINVAL;
+    if ((vel_ref == NULL) != (kl_out == NULL)) return OG_EINVAL;
+    const double two_pi = 6.283185307179586476925286766559;
+    #pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t i = 0; i < n; ++i) {
+        double sum_sq = 0.0, sum_kl = 0.0;
+        for (int64_t e = 0; e < d; ++e) {
+            double xe = (double)x[i * d + e];
+            double m = c_x * xe + c_v * load_vel(vel, vel_dtype, i * d + e);
+            double z = ((double)x_next[i * d + e] - m) / noise_std;
+            sum_sq += z * z;
+            if (vel_ref) {
+                double m_ref = c_x * xe + c_v * load_vel(vel_ref, vel_dtype, i * d + e);
+                double dm = m - m_ref;
+                sum_kl += dm * dm;
+            }
+        }
+        double lp = -0.5 * sum_sq - 0.5 * (double)d * log(two_pi * noise_std * noise_std);
+        double kl = sum_kl / (2.0 * noise_std * noise_std);
+        if (logp_mean) { lp /= (double)d; kl /= (double)d; }
+        logp_out[i] = lp;
+        if (kl_out) kl_out[i] = kl;
+    }
+    return OG_OK;
+}
+
+/*
+ * Clipped surrogate objective over T steps and n trajectories (Eq. "pro_grpo_method"):
+ *     r[t,i]   = exp(logp_new[t,i] - logp_old[t,i])                       (Eq. "ratio_method")
+ *     surr     = min( r A_i , clip(r, 1-eps, 1+eps) A_i )
+ *     J        = mean over (t,i) of ( surr - beta * kl[t,i] )
+ * Also the derivative dJ/dlogp_new[t,i]: (1/(nT)) * A_i * r where the unclipped branch is
+ * the active one (r A <= clip(r) A, which includes the whole interior of the clip range),
+ * else 0.  kl may be NULL (beta term dropped).
+ */
+int og_policy_objective(int64_t T, int64_t n, const double *logp_new, const double *logp_old,
+                        const double *kl, const double *adv, double clip_eps, double beta,
+                        double *ratio_out, double *dlogp_out, double *objective_out)
+{
+    if (T <= 0 || n <= 0 || !logp_new || !logp_old || !adv || !objective_out || !(clip_eps >= 0.0))
+        return OG_EINVAL;
+    double total = 0.0;
+    const double inv = 1.0 / ((double)T * (double)n);
+    for (int64_t t = 0; t < T; ++t)
+        for (int64_t i = 0; i < n; ++i) {
+            int64_t j = t * n + i;
+            double r = exp(logp_new[j] - logp_old[j]);
+            double lo = 1.0 - clip_eps, hi = 1.0 + clip_eps;
+            double rc = r < lo ? lo : (r > hi ? hi : r);
+            double a = adv[i];
+            double s1 = r * a, s2 = rc * a;
+            double surr = s1 < s2 ? s1 : s2;
+            total += surr - (kl ? beta * kl[j] : 0.0);
+            if (ratio_out) ratio_out[j] = r;
+            if (dlogp_out) dlogp_out[j] = (s1 <= s2) ? inv * a * r : 0.0;
+        }
+    *objective_out = total * inv;
+    return OG_OK;
+}
+
+/*
+ * Gradient of J with respect to the new prediction at one step, given dJ/dlogp of that step
+ * (dlogp[i]) and dJ/dkl (a scalar, -beta/(nT)):
+ *     dlogp/dvel_e = c_v (x_next_e - m_e) / s^2          (/ d if logp_mean)
+ *     dkl/dvel_e   = c_v^2 (vel_e - vel_ref_e) / s^2     (/ d if logp_mean)
+ */
+int og_policy_backward(int64_t n, int64_t d, const float *x, const float *x_next,
+                       const void *vel, const void *vel_ref, int vel_dtype,
+                       double c_x, double c_v, double noise_std, int logp_mean,
+                       const double *dlogp, double dkl, double *grad_out)
+{
+    if (n < 0 || d <= 0 || !x || !x_next || !vel || !dlogp || !grad_out || !(noise_std > 0.0))
+        return OG_EINVAL;
+    const double inv_s2 = 1.0 / (noise_std * noise_std);
+    const double scale = logp_mean ? 1.0 / (double)d : 1.0;
+    #pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t i = 0; i < n; ++i)
+        for (int64_t e = 0; e < d; ++e) {
+            double v = load_vel(vel, vel_dtype, i * d + e);
+            double m = c_x * (double)x[i * d + e] + c_v * v;
+            double g = dlogp[i] * c_v * ((double)x_next[i * d + e] - m) * inv_s2;
+            if (vel_ref)
+                g += dkl * c_v * c_v * (v - load_vel(vel_ref, vel_dtype, i * d + e)) * inv_s2;
+            grad_out[i * d + e] = g * scale;
+        }
+    return OG_OK;
 }
