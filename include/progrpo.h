@@ -183,6 +183,45 @@ int pg_advantages(pg_rollout *h, const float *rewards, float *adv, float *mean, 
                   void *stream);
 
 /*
+ * Policy update on the survivors, forward part for one step (Eq. "ratio_method": pi_theta is
+ * the Gaussian policy induced by Eq. "euler_method"; KL term of Eq. "pro_grpo_method").
+ * For each of the n_active rows, with m = c_x x + c_v vel and s = noise_std > 0:
+ *     logp_out[i] = -1/2 sum_e ((x_next_e - m_e)/s)^2 - d/2 ln(2 pi s^2)        (/ d if logp_mean)
+ *     kl_out[i]   = KL(N(m, s^2 I) || N(m_ref, s^2 I)) = c_v^2 sum_e (vel_e - vel_ref_e)^2 / (2 s^2)
+ *                                                                               (/ d if logp_mean)
+ * x, x_next [n_active, d] fp32: stored latents before / after the step; vel, vel_ref
+ * [n_active, d] in cfg.vel_dtype: new and reference predictions.  vel_ref and kl_out are
+ * both NULL or both given.  Read-only pass; uses the handle's reduction scratch (same stream
+ * rule as the other calls).  Does not move any cursor.
+ */
+int pg_policy_logprob(pg_rollout *h, const pg_step_coef *coef, const float *x, const float *x_next,
+                      const void *vel, const void *vel_ref, float *logp_out, float *kl_out, void *stream);
+
+/*
+ * Clipped surrogate objective of Eq. "pro_grpo_method" over n_steps steps and the n_active
+ * survivors: r = exp(logp_new - logp_old), surr = min(r A, clip(r, 1-clip_eps, 1+clip_eps) A),
+ * objective[0] = mean over (step, trajectory) of (surr - beta * kl).  logp_new, logp_old, kl
+ * (nullable), ratio (nullable, out), dlogp (out) are [n_steps, n_active] fp32; adv [n_active].
+ * dlogp = d objective / d logp_new: A r / (n_steps n_active) where the unclipped branch is
+ * active, else 0.  The matching derivative with respect to kl is the constant
+ * -beta / (n_steps n_active).  Evaluated in fp64 from the fp32 inputs; one small launch.
+ */
+int pg_policy_objective(pg_rollout *h, int32_t n_steps, const float *logp_new, const float *logp_old,
+                        const float *kl, const float *adv, float clip_eps, float beta, float *ratio,
+                        float *dlogp, float *objective, void *stream);
+
+/*
+ * Gradient of the objective with respect to the new prediction of one step:
+ *     grad_e = dlogp[i] * c_v (x_next_e - m_e) / s^2 + dkl * c_v^2 (vel_e - vel_ref_e) / s^2
+ * (both terms / d if logp_mean).  dlogp [n_active] is the row of pg_policy_objective's dlogp for
+ * this step, dkl the scalar -beta / (n_steps n_active) (ignored when vel_ref is NULL).
+ * grad_vel [n_active, d] in cfg.vel_dtype (bf16 rounded to nearest even).
+ */
+int pg_policy_backward(pg_rollout *h, const pg_step_coef *coef, const float *x, const float *x_next,
+                       const void *vel, const void *vel_ref, const float *dlogp, double dkl,
+                       void *grad_vel, void *stream);
+
+/*
  * Stateless OVF over many groups in one launch: selection as pg_prune_ovf for
  * n_groups groups of n scores, keeping k; optionally the kept scores and their
  * group-relative advantages (Eq. "advK" applied to the kept scores) in the

@@ -70,6 +70,9 @@ def lib() -> ctypes.CDLL:
     L.pg_prune_ovf.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     L.pg_compact.argtypes = [vp, vp, vp, vp, sz, vp]
     L.pg_advantages.argtypes = [vp, vp, vp, vp, vp, vp]
+    L.pg_policy_logprob.argtypes = [vp, ctypes.POINTER(StepCoef), vp, vp, vp, vp, vp, vp, vp]
+    L.pg_policy_objective.argtypes = [vp, i32, vp, vp, vp, vp, ctypes.c_float, ctypes.c_float, vp, vp, vp, vp]
+    L.pg_policy_backward.argtypes = [vp, ctypes.POINTER(StepCoef), vp, vp, vp, vp, vp, ctypes.c_double, vp, vp]
     L.pg_ovf_select_batched.argtypes = [i32, i32, i32, vp, vp, vp, vp, ctypes.c_float, vp, vp]
     L.pg_rollout_host_workspace_bytes.argtypes = [ctypes.POINTER(Config)]
     L.pg_rollout_host_workspace_bytes.restype = sz
@@ -87,7 +90,8 @@ def lib() -> ctypes.CDLL:
     for name in ("pg_rollout_init", "pg_rollout_destroy", "pg_rollout_reset", "pg_rollout_status",
                  "pg_step", "pg_score", "pg_prune_ovf", "pg_compact", "pg_advantages",
                  "pg_ovf_select_batched", "pg_rollout_host", "pg_rollout_traj_ids",
-                 "pg_philox_raw", "pg_normal_rows", "pg_score_static"):
+                 "pg_philox_raw", "pg_normal_rows", "pg_score_static", "pg_policy_logprob",
+                 "pg_policy_objective", "pg_policy_backward"):
         getattr(L, name).restype = ctypes.c_int
     _lib = L
     return L
@@ -179,6 +183,25 @@ def compact(h: int, keep_idx, src, dst, row_bytes: int, stream=None) -> None:
 def advantages(h: int, rewards, adv, mean=None, std=None, stream=None) -> None:
     _check(lib().pg_advantages(h, _p(rewards), _p(adv), _p(mean), _p(std), _stream(stream)),
            "pg_advantages")
+
+
+def policy_logprob(h: int, coef, x, x_next, vel, vel_ref, logp_out, kl_out=None, stream=None) -> None:
+    c = StepCoef(*coef)
+    _check(lib().pg_policy_logprob(h, ctypes.byref(c), _p(x), _p(x_next), _p(vel), _p(vel_ref),
+                                   _p(logp_out), _p(kl_out), _stream(stream)), "pg_policy_logprob")
+
+
+def policy_objective(h: int, n_steps: int, logp_new, logp_old, kl, adv, clip_eps: float, beta: float,
+                     ratio, dlogp, objective, stream=None) -> None:
+    _check(lib().pg_policy_objective(h, n_steps, _p(logp_new), _p(logp_old), _p(kl), _p(adv), clip_eps,
+                                     beta, _p(ratio), _p(dlogp), _p(objective), _stream(stream)),
+           "pg_policy_objective")
+
+
+def policy_backward(h: int, coef, x, x_next, vel, vel_ref, dlogp, dkl: float, grad_vel, stream=None) -> None:
+    c = StepCoef(*coef)
+    _check(lib().pg_policy_backward(h, ctypes.byref(c), _p(x), _p(x_next), _p(vel), _p(vel_ref),
+                                    _p(dlogp), dkl, _p(grad_vel), _stream(stream)), "pg_policy_backward")
 
 
 def ovf_select_batched(n_groups: int, n: int, k: int, scores, keep_idx, kept_scores=None, adv=None,

@@ -180,11 +180,57 @@ __device__ __forceinline__ void finish_row(float warp_total, int row, int chunk,
     tickets[row] = 0u;
   }
 }
+
+// Same reduction for NV sums per row at once (slot layout [row][chunk][NV]).
+template <int NV, typename Fin>
+__device__ __forceinline__ void finish_row_n(const float (&warp_total)[NV], int row, int chunk, int chunks,
+                                             float* partials, unsigned int* tickets, Fin fin) {
+  __shared__ float warp_part[NV][kRowWarps];
+  const int lane = threadIdx.x & 31;
+  if (lane == 0) {
+#pragma unroll
+    for (int j = 0; j < NV; ++j) warp_part[j][threadIdx.x >> 5] = warp_total[j];
+  }
+  __syncthreads();
+  if (threadIdx.x >= 32) return;
+  float v[NV];
+#pragma unroll
+  for (int j = 0; j < NV; ++j) v[j] = warp_sum(lane < kRowWarps ? warp_part[j][lane] : 0.f);
+  double s[NV];
+  if (chunks == 1) {
+#pragma unroll
+    for (int j = 0; j < NV; ++j) s[j] = (double)v[j];
+    if (lane == 0) fin(s);
+    return;
+  }
+  int last = 0;
+  if (lane == 0) {
+#pragma unroll
+    for (int j = 0; j < NV; ++j) partials[((size_t)row * chunks + chunk) * NV + j] = v[j];
+    __threadfence();
+    const unsigned int t = atomicAdd(&tickets[row], 1u);
+    last = (t == (unsigned int)chunks - 1u);
+  }
+  last = __shfl_sync(0xFFFFFFFFu, last, 0);
+  if (!last) return;
+  __threadfence();
+#pragma unroll
+  for (int j = 0; j < NV; ++j) {
+    double a = 0.0;
+    for (int c = lane; c < chunks; c += 32)
+      a += (double)__ldcg(&partials[((size_t)row * chunks + c) * NV + j]);
+    s[j] = warp_sum(a);
+  }
+  if (lane == 0) {
+    fin(s);
+    tickets[row] = 0u;
+  }
+}
 #endif
 
 // ---------------------------------------------------------------- launchers (device pointers)
 struct RowScratch {
-  float* partials;        // [rows * row_geometry(rows, elems).chunks]
+  float* partials;        // [rows * row_geometry(rows, elems).chunks * sums per row (1 or 2)]
   unsigned int* tickets;  // [rows], zero between launches
 };
 
@@ -196,6 +242,20 @@ int launch_step(int n_rows, int elems, int vel_dtype, const float* x_in, const v
 int launch_score(int n_rows, int elems, int vel_dtype, const float* x, const void* vel,
                  double p_x, double p_v, float* scores_out, float* preview_out,
                  RowScratch scratch, cudaStream_t stream, int forced_chunk_quads = 0);
+
+int launch_policy_logprob(int n_rows, int elems, int vel_dtype, const float* x, const float* x_next,
+                          const void* vel, const void* vel_ref, double c_x, double c_v,
+                          double noise_std, int logp_mean, float* logp_out, float* kl_out,
+                          RowScratch scratch, cudaStream_t stream);
+
+int launch_policy_objective(int n_steps, int n_rows, const float* logp_new, const float* logp_old,
+                            const float* kl, const float* adv, float clip_eps, float beta,
+                            float* ratio, float* dlogp, float* objective, cudaStream_t stream);
+
+int launch_policy_backward(int n_rows, int elems, int vel_dtype, const float* x, const float* x_next,
+                           const void* vel, const void* vel_ref, double c_x, double c_v,
+                           double noise_std, int logp_mean, const float* dlogp, double dkl,
+                           void* grad_vel, cudaStream_t stream);
 
 int launch_ovf(int n_groups, int n, int k, const float* scores, int32_t* keep_idx,
                int32_t* src_rows, float* sel_var, float* kept_scores, float* adv, float adv_eps,

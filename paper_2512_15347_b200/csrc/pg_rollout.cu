@@ -90,7 +90,7 @@ int pg_rollout_init(const pg_config* cfg, pg_rollout** out) {
   cudaError_t e = cudaGetDevice(&h->device);
   if (e == cudaSuccess) e = cudaMalloc(&h->d_traj[0], rows * sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMalloc(&h->d_traj[1], rows * sizeof(int32_t));
-  if (e == cudaSuccess) e = cudaMalloc(&h->d_partials, slots * sizeof(float));
+  if (e == cudaSuccess) e = cudaMalloc(&h->d_partials, 2 * slots * sizeof(float))   /* up to two sums per row */;
   if (e == cudaSuccess) e = cudaMalloc(&h->d_tickets, rows * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMalloc(&h->d_status, sizeof(int32_t));
   if (e == cudaSuccess) e = cudaMemset(h->d_tickets, 0, rows * sizeof(unsigned int));
@@ -212,6 +212,44 @@ int pg_advantages(pg_rollout* h, const float* rewards, float* adv, float* mean, 
   if (!h || !rewards || !adv) return PG_EINVAL;
   return pg::launch_advantages(h->cfg.n_groups, h->k_cur, rewards, h->cfg.adv_eps, adv, mean, std,
                                (cudaStream_t)stream);
+}
+
+int pg_policy_logprob(pg_rollout* h, const pg_step_coef* coef, const float* x, const float* x_next,
+                      const void* vel, const void* vel_ref, float* logp_out, float* kl_out, void* stream) {
+  if (!h || !coef || !x || !x_next || !vel || !logp_out) return PG_EINVAL;
+  if ((vel_ref == nullptr) != (kl_out == nullptr)) return PG_EINVAL;
+  if (!aligned16(x) || !aligned16(x_next) || !aligned16(vel) || !aligned16(vel_ref)) return PG_EINVAL;
+  if (!(coef->noise_std > 0.0) || !std::isfinite(coef->c_x) || !std::isfinite(coef->c_v) ||
+      !std::isfinite(coef->noise_std))
+    return PG_EINVAL;
+  pg::RowScratch scratch{h->d_partials, h->d_tickets};
+  return pg::launch_policy_logprob(h->cfg.n_groups * h->k_cur, h->cfg.elems, h->cfg.vel_dtype, x, x_next,
+                                   vel, vel_ref, coef->c_x, coef->c_v, coef->noise_std,
+                                   h->cfg.logp_mean, logp_out, kl_out, scratch, (cudaStream_t)stream);
+}
+
+int pg_policy_objective(pg_rollout* h, int32_t n_steps, const float* logp_new, const float* logp_old,
+                        const float* kl, const float* adv, float clip_eps, float beta, float* ratio,
+                        float* dlogp, float* objective, void* stream) {
+  if (!h || n_steps < 1 || !logp_new || !logp_old || !adv || !dlogp || !objective) return PG_EINVAL;
+  if (!(clip_eps >= 0.f) || !std::isfinite(beta)) return PG_EINVAL;
+  return pg::launch_policy_objective(n_steps, h->cfg.n_groups * h->k_cur, logp_new, logp_old, kl, adv,
+                                     clip_eps, beta, ratio, dlogp, objective, (cudaStream_t)stream);
+}
+
+int pg_policy_backward(pg_rollout* h, const pg_step_coef* coef, const float* x, const float* x_next,
+                       const void* vel, const void* vel_ref, const float* dlogp, double dkl,
+                       void* grad_vel, void* stream) {
+  if (!h || !coef || !x || !x_next || !vel || !dlogp || !grad_vel) return PG_EINVAL;
+  if (!aligned16(x) || !aligned16(x_next) || !aligned16(vel) || !aligned16(vel_ref) ||
+      !aligned16(grad_vel))
+    return PG_EINVAL;
+  if (!(coef->noise_std > 0.0) || !std::isfinite(coef->c_x) || !std::isfinite(coef->c_v) ||
+      !std::isfinite(coef->noise_std) || !std::isfinite(dkl))
+    return PG_EINVAL;
+  return pg::launch_policy_backward(h->cfg.n_groups * h->k_cur, h->cfg.elems, h->cfg.vel_dtype, x, x_next,
+                                    vel, vel_ref, coef->c_x, coef->c_v, coef->noise_std,
+                                    h->cfg.logp_mean, dlogp, dkl, grad_vel, (cudaStream_t)stream);
 }
 
 int pg_ovf_select_batched(int32_t n_groups, int32_t n, int32_t k, const float* scores,

@@ -1,0 +1,127 @@
+"""GPU parity of the policy-update calls (log-prob of stored transitions + KL, clipped
+surrogate objective, gradient w.r.t. the prediction) against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2512_15347_b200 import workloads as wl
+from tests import util as U
+
+pytestmark = pytest.mark.gpu
+
+
+def grad_err(a, b) -> float:
+    """max_e |a-b| / max(|b_e|, rms(b_row))"""
+    return U.latent_err(a, b)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("d", [4, 1000, 3 * 8192 + 20, 65536])
+@pytest.mark.parametrize("logp_mean", [False, True])
+def test_policy_update_matches_oracle(bf16, d, logp_mean):
+    from paper_2512_15347_b200 import binding as B
+    G, K, T = 3, 4, 3
+    n = G * K
+    rng = np.random.default_rng(d + 7 * bf16 + logp_mean)
+    coef = (1.0, 0.1, 0.25)
+    vd = B.VEL_BF16 if bf16 else B.VEL_F32
+    h = B.rollout_init(B.make_config(G, K, d, T, [], 3, vd, logp_mean=logp_mean))
+
+    def vel(arr):
+        t = torch.from_numpy(arr.astype(np.float32))
+        return wl.as_numpy_velocity(t.to(torch.bfloat16) if bf16 else t)
+
+    try:
+        xs = [rng.standard_normal((n, d)).astype(np.float32) for _ in range(T)]
+        v_old = [vel(rng.standard_normal((n, d))) for _ in range(T)]
+        # new prediction close to the old one so that ratios stay finite in sum mode
+        delta = 2e-3 if not logp_mean else 0.5
+        v_new, xn = [], []
+        for t in range(T):
+            vo = U.vel_to_dev(v_old[t]).float().cpu().numpy()
+            v_new.append(vel(vo + delta * rng.standard_normal((n, d))))
+            xn.append((xs[t] + coef[1] * vo + coef[2] * rng.standard_normal((n, d))).astype(np.float32))
+        adv = rng.standard_normal(n).astype(np.float32)
+        lp_old = np.stack([oracle.policy_logprob(xs[t], xn[t], v_old[t], None, *coef, logp_mean)[0]
+                           for t in range(T)]).astype(np.float32)
+
+        lp_new = torch.empty(T, n, device="cuda")
+        kl = torch.empty(T, n, device="cuda")
+        dev = [(U.to_dev(xs[t]), U.to_dev(xn[t]), U.vel_to_dev(v_new[t]), U.vel_to_dev(v_old[t]))
+               for t in range(T)]
+        ref_lp, ref_kl = [], []
+        for t in range(T):
+            B.policy_logprob(h, coef, dev[t][0], dev[t][1], dev[t][2], dev[t][3], lp_new[t], kl[t])
+            a, b = oracle.policy_logprob(xs[t], xn[t], v_new[t], v_old[t], *coef, logp_mean)
+            ref_lp.append(a)
+            ref_kl.append(b)
+        scale = 1.0 if logp_mean else d
+        got_lp = lp_new.cpu().numpy()
+        assert (np.abs(got_lp - np.stack(ref_lp)) / np.maximum(np.abs(np.stack(ref_lp)), 0.5 * scale)).max() <= 1e-5
+        np.testing.assert_allclose(kl.cpu().numpy(), np.stack(ref_kl), rtol=1e-5, atol=1e-30)
+        # without a reference the log-prob is unchanged
+        lp_only = torch.empty(n, device="cuda")
+        B.policy_logprob(h, coef, dev[0][0], dev[0][1], dev[0][2], None, lp_only, None)
+        assert torch.equal(lp_only, lp_new[0])
+
+        # objective from the device's own fp32 log-probs
+        ratio = torch.empty(T, n, device="cuda")
+        dlogp = torch.empty(T, n, device="cuda")
+        obj = torch.empty(1, device="cuda")
+        B.policy_objective(h, T, lp_new, U.to_dev(lp_old), kl, U.to_dev(adv), 0.2, 0.3, ratio, dlogp, obj)
+        ref_obj, ref_ratio, ref_dlogp = oracle.policy_objective(got_lp, lp_old, kl.cpu().numpy(), adv, 0.2, 0.3)
+        np.testing.assert_allclose(ratio.cpu().numpy(), ref_ratio, rtol=1e-6)
+        np.testing.assert_allclose(dlogp.cpu().numpy(), ref_dlogp, rtol=1e-6, atol=1e-30)
+        assert float(obj.item()) == pytest.approx(ref_obj, rel=1e-5, abs=1e-7)
+
+        # gradient for every step
+        dkl = -0.3 / (T * n)
+        for t in range(T):
+            g = torch.empty(n, d, device="cuda", dtype=torch.bfloat16 if bf16 else torch.float32)
+            B.policy_backward(h, coef, dev[t][0], dev[t][1], dev[t][2], dev[t][3], dlogp[t], dkl, g)
+            ref_g = oracle.policy_backward(xs[t], xn[t], v_new[t], v_old[t], *coef,
+                                           dlogp[t].cpu().numpy().astype(np.float64), dkl, logp_mean)
+            tol = 2.0 ** -8 if bf16 else 1e-5
+            assert grad_err(g.float().cpu().numpy(), ref_g) <= tol
+    finally:
+        torch.cuda.synchronize()
+        B.rollout_destroy(h)
+
+
+def test_policy_update_after_a_rollout_has_unit_ratio():
+    """Re-evaluating the rollout's own predictions gives back its log-probs: ratio 1, objective =
+    mean advantage = 0, and the objective's gradient is A / (nT) * dlogp/dv."""
+    from paper_2512_15347_b200 import binding as B
+    from paper_2512_15347_b200.rollout import Rollout
+    w = wl.Workload("upd", 4, 8, (), 3, 8192 + 512, 1, "bf16", 5, "normal", "preview")
+    inp = U.SharedInputs(w)
+    ro = Rollout(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, torch.bfloat16, logp_mean=True)
+    xs = [U.to_dev(inp.x0)]
+    vels = []
+
+    def velocity(s, x):
+        v = inp.vel_device(s, x)
+        vels.append(v)
+        if s > 0:
+            xs.append(x.clone())
+        return v
+
+    out = ro.run(xs[0], w.step_coef, w.preview_coef, velocity)
+    xs.append(out.x_final.clone())
+    n, T = w.n_groups * w.n_expand, w.n_steps
+    lp_new = torch.empty(T, n, device="cuda")
+    for t in range(T):
+        B.policy_logprob(ro.h, w.step_coef(t), xs[t], xs[t + 1], vels[t], None, lp_new[t], None)
+    lp_old = torch.stack(out.logp)
+    torch.cuda.synchronize()
+    # fp32 storage of x_{t+1} perturbs the recomputed mean log-prob by ~1e-7
+    assert (lp_new - lp_old).abs().max().item() < 2e-6
+    ratio = torch.empty(T, n, device="cuda")
+    dlogp = torch.empty(T, n, device="cuda")
+    obj = torch.empty(1, device="cuda")
+    B.policy_objective(ro.h, T, lp_new, lp_old, None, out.adv, 0.2, 0.0, ratio, dlogp, obj)
+    torch.cuda.synchronize()
+    assert (ratio - 1).abs().max().item() < 1e-5
+    assert abs(obj.item()) < 1e-6
+    ro.close()
