@@ -316,6 +316,38 @@ def run_ours(args):
                "workload": f"{m['n_groups']} groups x {m['n']} scores -> {m['k']} (select + index/score "
                            "compaction + advantages), L2 flushed between repetitions"}
 
+    # policy-update kernels on the survivors' shape (secondary numbers; not part of `value`)
+    policy = None
+    if rank == 0 and w.vel_dtype == "bf16" and w.velocity == "normal":
+        rows = w.n_groups * w.final_keep
+        xa, xb = ro.x[0][:rows], ro.x[1][:rows]
+        va, vb = vels[-1][:rows], vels[-2][:rows]
+        lp = torch.empty(rows, device=dev)
+        klv = torch.empty(rows, device=dev)
+        dl = torch.full((rows,), 1e-3, device=dev)
+        grad = torch.empty(rows, w.elems, device=dev, dtype=torch.bfloat16)
+        coef = w.step_coef(0)
+
+        def timed(fn, reps=10):
+            ts = []
+            for i in range(reps + 3):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                fn()
+                b.record()
+                torch.cuda.synchronize()
+                if i >= 3:
+                    ts.append(a.elapsed_time(b))
+            ts.sort()
+            return ts[len(ts) // 2]
+        t_lp = timed(lambda: B.policy_logprob(ro.h, coef, xa, xb, va, vb, lp, klv))
+        t_bw = timed(lambda: B.policy_backward(ro.h, coef, xa, xb, va, vb, dl, -1e-6, grad))
+        policy = {"rows": rows, "logprob_kl_gbs": rows * w.elems * 12 / (t_lp * 1e-3) / 1e9,
+                  "backward_gbs": rows * w.elems * 14 / (t_bw * 1e-3) / 1e9,
+                  "bytes_per_element": {"logprob_kl": 12, "backward": 14},
+                  "note": "per-step kernels of the update on the survivors (x, x_next fp32; new and "
+                          "reference predictions bf16; bf16 gradient), inputs larger than L2"}
+
     # end to end through the host-buffer entry point (pinned host memory, copies inside the timing)
     e2e = None
     if not args.no_e2e:
@@ -342,7 +374,7 @@ def run_ours(args):
                                 v["launches"] // args.steps} for k, v in kinds.items()},
                 "score_gbs": score_gbs, "prune_stage_gbs": prune_stage_gbs,
                 "hbm_gbs_whole_rollout": (step_bytes + (score_bytes if score_gbs else 0)) / (total_ms * 1e-3) / 1e9,
-                "ovf_microbench": ovf, "e2e": e2e, "cpu_baseline": cpu_base}
+                "ovf_microbench": ovf, "policy_update": policy, "e2e": e2e, "cpu_baseline": cpu_base}
         print(json.dumps(line))
     ro.close()
     if dist is not None:
