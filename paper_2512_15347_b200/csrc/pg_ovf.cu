@@ -246,11 +246,18 @@ ovf_select_kernel(const __grid_constant__ OvfParams p) {
 
 // ---------------------------------------------------------------- groups of up to 256 scores
 //
-// One warp per group, E = 1, 2, 4 or 8 scores per lane (n <= 32 * E).  The 64-bit keys are
-// sorted with a bitonic network held in registers (exchanges inside a lane for distances
-// below E, warp shuffles above); slots >= n hold an all-ones key and sort to the end.  Since
-// keys are distinct any correct sorting network yields the same order as the counting kernel.
-// No CTA barrier is used: warps of a CTA are independent.
+// One warp per group, E = 1, 2, 4 or 8 scores per lane (n <= 32 * E), no CTA barrier.
+//  1. The 32-bit order keys alone are sorted with a bitonic network held in registers (one
+//     integer min and one max per compare-exchange; shuffles for distances of E and more).
+//     Slots >= n hold an all-ones key and sort to the end.
+//  2. Each element finds its rank in the total order (score, slot) by a binary search for its
+//     key in the sorted list; where equal keys exist (rare for real scores) the rank is advanced
+//     by the number of equal keys in lower slots, counted directly.  Ranks are a permutation.
+//  3. Running sums from both ends: the centred values and their squares are formed by all lanes
+//     in parallel, then lanes 0 and 1 accumulate them serially, in order, in fp64 with explicitly
+//     rounded operations - the same operations in the same order as a plain serial loop.
+//  4. k+1 candidates, argmax with the "largest j" tie rule, membership by rank; every lane holds
+//     its scores in slot order, so a popcount prefix over lanes gives ascending slot order.
 constexpr int kOvfWarpsPerCta = 4;
 
 __device__ __forceinline__ float key_to_score(uint32_t key) {
@@ -267,18 +274,18 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int g = blockIdx.x * kOvfWarpsPerCta + warp;
   if (g >= n_groups) return;
-  const size_t per_warp = (size_t)(k + 1) * 4 * sizeof(double) + (size_t)N * sizeof(float) + 32;
+  const size_t per_warp = (size_t)(k + 1) * 4 * sizeof(double) + (size_t)N * 2 * sizeof(uint32_t);
   unsigned char* base = smem + (size_t)warp * per_warp;
   double* L1 = reinterpret_cast<double*>(base);
   double* L2 = L1 + (k + 1);
   double* H1 = L2 + (k + 1);
   double* H2 = H1 + (k + 1);
-  float* sorted = reinterpret_cast<float*>(H2 + (k + 1));
-  unsigned int* mask = reinterpret_cast<unsigned int*>(sorted + N);     // N bits, 8 words
+  uint32_t* skey = reinterpret_cast<uint32_t*>(H2 + (k + 1));   // [N] sorted keys
+  uint32_t* okey = skey + N;                                    // [N] keys in slot order
 
   const float* sc = p.scores + (size_t)g * n;
   float orig[E];
-  unsigned long long key[E];
+  uint32_t mine[E], key[E];
   bool bad = false;
 #pragma unroll
   for (int r = 0; r < E; ++r) {
@@ -286,55 +293,48 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
     if (i < n) {
       orig[r] = sc[i];
       bad |= !(fabsf(orig[r]) <= FLT_MAX);
-      key[r] = ((unsigned long long)order_key(orig[r]) << 32) | (unsigned int)i;
+      mine[r] = order_key(orig[r]);
     } else {
       orig[r] = 0.f;
-      key[r] = ~0ull;
+      mine[r] = 0xFFFFFFFFu;
     }
+    key[r] = mine[r];
+    okey[i] = mine[r];
   }
   if (bad && p.status) atomicOr(p.status, 1);
-  if (lane < 8) mask[lane] = 0u;
 
-  // Bitonic sort, ascending over index lane * E + r, in the form whose compare-exchanges all
-  // point the same way: each merge of two sorted runs of length size/2 first pairs i with its
-  // mirror i ^ (size - 1), then halves the distance; the lower index always keeps the minimum.
+  // 1. bitonic sort, ascending over index lane * E + r; every compare-exchange points the same
+  //    way: a merge first pairs i with its mirror i ^ (size - 1), then halves the distance.
 #pragma unroll
   for (int size = 2; size <= N; size <<= 1) {
-    // mirror step
     if (size <= E) {
 #pragma unroll
       for (int r = 0; r < E; ++r) {
         const int q = r ^ (size - 1);
         if (r < q) {
-          const unsigned long long a = key[r], b = key[q];
-          const bool swap = a > b;
-          key[r] = swap ? b : a;
-          key[q] = swap ? a : b;
+          const uint32_t a = key[r], b = key[q];
+          key[r] = min(a, b);
+          key[q] = max(a, b);
         }
       }
     } else {
       const int lane_mask = size / E - 1;
       const bool lower = (lane & (size / E / 2)) == 0;
-      unsigned long long other[E];
+      uint32_t other[E];
 #pragma unroll
       for (int r = 0; r < E; ++r) other[r] = __shfl_xor_sync(0xFFFFFFFFu, key[r ^ (E - 1)], lane_mask);
 #pragma unroll
-      for (int r = 0; r < E; ++r) {
-        const bool other_smaller = other[r] < key[r];
-        key[r] = (lower == other_smaller) ? other[r] : key[r];
-      }
+      for (int r = 0; r < E; ++r) key[r] = lower ? min(key[r], other[r]) : max(key[r], other[r]);
     }
-    // halving steps
 #pragma unroll
     for (int j = size >> 2; j > 0; j >>= 1) {
       if (j < E) {
 #pragma unroll
         for (int r = 0; r < E; ++r) {
           if ((r & j) == 0) {
-            const unsigned long long a = key[r], b = key[r | j];
-            const bool swap = a > b;
-            key[r] = swap ? b : a;
-            key[r | j] = swap ? a : b;
+            const uint32_t a = key[r], b = key[r | j];
+            key[r] = min(a, b);
+            key[r | j] = max(a, b);
           }
         }
       } else {
@@ -342,36 +342,63 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
         const bool lower = (lane & lane_mask) == 0;
 #pragma unroll
         for (int r = 0; r < E; ++r) {
-          const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, key[r], lane_mask);
-          const bool other_smaller = other < key[r];
-          key[r] = (lower == other_smaller) ? other : key[r];
+          const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, key[r], lane_mask);
+          key[r] = lower ? min(key[r], other) : max(key[r], other);
         }
       }
     }
   }
 #pragma unroll
-  for (int r = 0; r < E; ++r) sorted[lane * E + r] = key_to_score((uint32_t)(key[r] >> 32));
+  for (int r = 0; r < E; ++r) skey[lane * E + r] = key[r];
   __syncwarp();
 
-  // running sums from both ends, serial and in order (fp64, explicitly rounded)
+  // 2. rank of every own element in the order (score, slot)
+  int rank[E];
+#pragma unroll
+  for (int r = 0; r < E; ++r) {
+    int pos = 0;
+#pragma unroll
+    for (int step = N / 2; step > 0; step >>= 1)
+      if (skey[pos + step - 1] < mine[r]) pos += step;
+    rank[r] = pos;                                  // first position whose key is >= mine
+  }
+#pragma unroll
+  for (int r = 0; r < E; ++r) {
+    const int i = lane * E + r;
+    if (i < n && rank[r] + 1 < N && skey[rank[r] + 1] == mine[r]) {   // equal keys exist
+      int lower_slots = 0;
+      for (int j = 0; j < i; ++j) lower_slots += (okey[j] == mine[r]) ? 1 : 0;
+      rank[r] += lower_slots;
+    }
+  }
+
+  // 3. centred values and squares in parallel, then the serial running sums
+  const double pivot = arithmetic_value(key_to_score(skey[n / 2]));
+  for (int j = lane; j < k; j += 32) {
+    const double cl = __dsub_rn(arithmetic_value(key_to_score(skey[j])), pivot);
+    const double ch = __dsub_rn(arithmetic_value(key_to_score(skey[n - 1 - j])), pivot);
+    L1[j + 1] = cl;
+    L2[j + 1] = __dmul_rn(cl, cl);
+    H1[j + 1] = ch;
+    H2[j + 1] = __dmul_rn(ch, ch);
+  }
+  __syncwarp();
   if (lane < 2) {
-    const double pivot = arithmetic_value(sorted[n / 2]);
-    double a1 = 0.0, a2 = 0.0;
     double* S1 = lane == 0 ? L1 : H1;
     double* S2 = lane == 0 ? L2 : H2;
+    double a1 = 0.0, a2 = 0.0;
     S1[0] = 0.0;
     S2[0] = 0.0;
     for (int j = 1; j <= k; ++j) {
-      const int pos = lane == 0 ? (j - 1) : (n - j);
-      const double c = __dsub_rn(arithmetic_value(sorted[pos]), pivot);
-      a1 = __dadd_rn(a1, c);
-      a2 = __dadd_rn(a2, __dmul_rn(c, c));
+      a1 = __dadd_rn(a1, S1[j]);
+      a2 = __dadd_rn(a2, S2[j]);
       S1[j] = a1;
       S2[j] = a2;
     }
   }
   __syncwarp();
 
+  // 4. candidates
   double best_m = -1.0;
   int best_j = -1;
   for (int j = lane; j <= k; j += 32) {
@@ -392,18 +419,10 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
   const int high_from = n - (k - jstar);
   if (lane == 0 && p.sel_var) p.sel_var[g] = (float)(best_m / ((double)k * (double)k));
 
-  // kept slots as a bit set, then ascending slot order by popcount prefix
+  unsigned int bits = 0u;
 #pragma unroll
-  for (int r = 0; r < E; ++r) {
-    const int pos = lane * E + r;
-    if (pos < n && (pos < jstar || pos >= high_from)) {
-      const unsigned int slot = (unsigned int)key[r];
-      atomicOr(&mask[slot >> 5], 1u << (slot & 31));
-    }
-  }
-  __syncwarp();
-  const int first = lane * E;
-  const unsigned int bits = (mask[first >> 5] >> (first & 31)) & ((E == 32) ? 0xFFFFFFFFu : ((1u << E) - 1u));
+  for (int r = 0; r < E; ++r)
+    if (lane * E + r < n && (rank[r] < jstar || rank[r] >= high_from)) bits |= 1u << r;
   const int cnt = __popc(bits);
   int incl = cnt;
 #pragma unroll
@@ -411,6 +430,7 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
     const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
     if (lane >= o) incl += t;
   }
+  const int first = lane * E;
   int pos = incl - cnt;
   double sum_kept = 0.0;
 #pragma unroll
@@ -448,7 +468,7 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
 
 template <int E>
 static void launch_ovf_warp(const OvfParams& p, int n_groups, cudaStream_t stream) {
-  const size_t per_warp = (size_t)(p.k + 1) * 4 * sizeof(double) + (size_t)(32 * E) * sizeof(float) + 32;
+  const size_t per_warp = (size_t)(p.k + 1) * 4 * sizeof(double) + (size_t)(32 * E) * 2 * sizeof(uint32_t);
   const int ctas = (n_groups + kOvfWarpsPerCta - 1) / kOvfWarpsPerCta;
   ovf_warp_kernel<E><<<ctas, kOvfWarpsPerCta * 32, per_warp * kOvfWarpsPerCta, stream>>>(p, n_groups);
 }
