@@ -64,7 +64,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -140,10 +140,11 @@ def run_reference(args):
     import oracle
     from paper_2512_15347_b200 import workloads as wl
     w = wl.WORKLOADS[args.workload]
-    sample = OracleSample(w, min(ORACLE_GROUPS, w.n_groups))
     small = OracleSample(w, 1)
-    for _ in range(max(args.warmup, 0)):
-        small.run()
+    t1 = min([small.run() for _ in range(max(args.warmup, 1))])
+    # bounded sample: as many groups (up to ORACLE_GROUPS) as keep the timed steps near two minutes
+    groups = max(1, min(ORACLE_GROUPS, w.n_groups, int(120.0 / (max(args.steps, 1) * t1))))
+    sample = small if groups == 1 else OracleSample(w, groups)
     times = [sample.run() for _ in range(args.steps)]
     mean_sec = sum(times) / len(times)
     value = sample.sw.traj_steps / mean_sec
@@ -440,7 +441,7 @@ def run_e2e(B, wl, w, wr, rank, dist, dev, args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="large", choices=["large", "sd3", "sd15", "tiny"])
