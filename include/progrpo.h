@@ -164,6 +164,25 @@ int pg_prune_ovf(pg_rollout *h, int32_t stage, const float *scores, int32_t *kee
                  int32_t *src_rows, float *sel_var, void *stream);
 
 /*
+ * Uniform-subsampling baseline (Section 4.1, Fig. 1b: "uniformly subsampling k < G candidates"):
+ * same contract and cursor effects as pg_prune_ovf, but the k survivors of each group are a
+ * uniformly random subset, independent of any score.  Reproducible: slot i of group g draws the
+ * first Philox4x32-10 word of counter (i, stage, group_offset + g, stream id 4) under the
+ * handle's seed, and the k slots with the smallest (word, slot) are kept, in ascending slot order.
+ */
+int pg_prune_uniform(pg_rollout *h, int32_t stage, int32_t *keep_idx, int32_t *src_rows, void *stream);
+
+/*
+ * Reward-clustering diagnostics (Section 4.1): for each of n_groups groups of n scores the mean
+ * mu_G, the population standard deviation sigma_G and the fraction of the group inside the
+ * clustered region C_delta = { i : |R_i - mu_G| <= delta * sigma_G } (Eq. "near-mean").
+ * scores [n_groups * n] fp32; mean, std, clustered_frac (each nullable) [n_groups] fp32.
+ * Stateless; fp64 statistics.
+ */
+int pg_group_stats(int32_t n_groups, int32_t n, const float *scores, float delta, float *mean,
+                   float *std, float *clustered_frac, void *stream);
+
+/*
  * Survivor compaction of a caller-side row array after the most recent
  * pg_prune_ovf (Section 5.1: pruned trajectories "incur no further SDE
  * steps"): dst row g*k + p = src row g*K_prev + keep_idx[g*k + p]; order and

@@ -364,3 +364,28 @@ def policy_backward(x: np.ndarray, x_next: np.ndarray, vel: np.ndarray, vel_ref:
                                     _ptr(grad))
     _check(rc, "policy_backward")
     return grad
+
+
+# ---------------------------------------------------------------- diagnostics / uniform baseline
+
+def group_stats(scores: np.ndarray, delta: float):
+    """(mean, population std, fraction inside |R - mu| <= delta sigma) per group of [G, n] scores."""
+    scores = np.ascontiguousarray(scores, dtype=np.float32)
+    g, n = scores.shape
+    mean = np.empty(g)
+    std = np.empty(g)
+    frac = np.empty(g)
+    rc = _load().og_group_stats(ctypes.c_int(g), ctypes.c_int(n), _ptr(scores), ctypes.c_double(delta),
+                                _ptr(mean), _ptr(std), _ptr(frac))
+    _check(rc, "group_stats")
+    return mean, std, frac
+
+
+def select_uniform(n_groups: int, n: int, k: int, seed: int, stage: int, group_offset: int = 0) -> np.ndarray:
+    """Reproducible uniform k-of-n subsampling per group; int32 [G, k], ascending slots."""
+    keep = np.zeros((n_groups, k), dtype=np.int32)
+    rc = _load().og_select_uniform(ctypes.c_int(n_groups), ctypes.c_int(n), ctypes.c_int(k),
+                                   ctypes.c_uint64(seed), ctypes.c_uint32(stage),
+                                   ctypes.c_uint32(group_offset), _ptr(keep))
+    _check(rc, "select_uniform")
+    return keep

@@ -584,3 +584,68 @@ int og_policy_backward(int64_t n, int64_t d, const float *x, const float *x_next
         }
     return OG_OK;
 }
+
+/* ------------------------------------------------------------------ */
+/* Diagnostics and the uniform-subsampling baseline (Section 4)        */
+/* ------------------------------------------------------------------ */
+
+/*
+ * Reward-clustering diagnostics per group (Section 4.1): mean mu_G, population standard
+ * deviation sigma_G and the fraction of the group inside the clustered region
+ *     C_delta = { i : |R_i - mu_G| <= delta * sigma_G }          (Eq. "near-mean").
+ */
+int og_group_stats(int n_groups, int n, const float *scores, double delta,
+                   double *mean_out, double *std_out, double *clustered_out)
+{
+    if (n_groups < 0 || n < 1 || !scores || !(delta >= 0.0)) return OG_EINVAL;
+    for (int g = 0; g < n_groups; ++g) {
+        const float *r = scores + (size_t)g * n;
+        double mu = 0.0;
+        for (int i = 0; i < n; ++i) mu += (double)r[i];
+        mu /= (double)n;
+        double acc = 0.0;
+        for (int i = 0; i < n; ++i) { double dl = (double)r[i] - mu; acc += dl * dl; }
+        double sigma = sqrt(acc / (double)n);
+        int inside = 0;
+        for (int i = 0; i < n; ++i) if (fabs((double)r[i] - mu) <= delta * sigma) ++inside;
+        if (mean_out) mean_out[g] = mu;
+        if (std_out) std_out[g] = sigma;
+        if (clustered_out) clustered_out[g] = (double)inside / (double)n;
+    }
+    return OG_OK;
+}
+
+/*
+ * Uniform subsampling of k of n trajectories per group (the baseline of Section 4.1 and
+ * Fig. 1b), made reproducible with the counter-based generator: slot i of group `group`
+ * draws the word r_i = first output word of Philox4x32-10 with counter
+ * (i, stage, group, stream 4) and the seed as key; the k slots with the smallest (r_i, i)
+ * are kept and reported in ascending slot order.  Distinct words are equally likely to
+ * fall in any order, so every k-subset is equally likely.
+ */
+int og_select_uniform(int n_groups, int n, int k, uint64_t seed, uint32_t stage,
+                      uint32_t group_offset, int32_t *keep_idx)
+{
+    if (n_groups < 0 || n < 1 || k < 1 || k > n || !keep_idx) return OG_EINVAL;
+    uint32_t *word = (uint32_t *)malloc((size_t)n * sizeof(uint32_t));
+    if (!word) return OG_EINVAL;
+    uint32_t key[2] = { (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32) };
+    for (int g = 0; g < n_groups; ++g) {
+        for (int i = 0; i < n; ++i) {
+            uint32_t ctr[4] = { (uint32_t)i, stage, group_offset + (uint32_t)g, 4u };
+            uint32_t out[4];
+            og_philox4x32_10(ctr, key, out);
+            word[i] = out[0];
+        }
+        int w = 0;
+        for (int i = 0; i < n; ++i) {
+            int smaller = 0;
+            for (int j = 0; j < n; ++j)
+                if (word[j] < word[i] || (word[j] == word[i] && j < i)) ++smaller;
+            if (smaller < k) keep_idx[(size_t)g * k + w++] = i;
+        }
+        if (w != k) { free(word); return OG_EINVAL; }
+    }
+    free(word);
+    return OG_OK;
+}

@@ -68,6 +68,8 @@ def lib() -> ctypes.CDLL:
     L.pg_step.argtypes = [vp, i32, ctypes.POINTER(StepCoef), vp, vp, vp, vp, vp, vp]
     L.pg_score.argtypes = [vp, ctypes.POINTER(PreviewCoef), vp, vp, vp, vp, vp]
     L.pg_prune_ovf.argtypes = [vp, i32, vp, vp, vp, vp, vp]
+    L.pg_prune_uniform.argtypes = [vp, i32, vp, vp, vp]
+    L.pg_group_stats.argtypes = [i32, i32, vp, ctypes.c_float, vp, vp, vp, vp]
     L.pg_compact.argtypes = [vp, vp, vp, vp, sz, vp]
     L.pg_advantages.argtypes = [vp, vp, vp, vp, vp, vp]
     L.pg_policy_logprob.argtypes = [vp, ctypes.POINTER(StepCoef), vp, vp, vp, vp, vp, vp, vp]
@@ -91,7 +93,7 @@ def lib() -> ctypes.CDLL:
                  "pg_step", "pg_score", "pg_prune_ovf", "pg_compact", "pg_advantages",
                  "pg_ovf_select_batched", "pg_rollout_host", "pg_rollout_traj_ids",
                  "pg_philox_raw", "pg_normal_rows", "pg_score_static", "pg_policy_logprob",
-                 "pg_policy_objective", "pg_policy_backward"):
+                 "pg_policy_objective", "pg_policy_backward", "pg_prune_uniform", "pg_group_stats"):
         getattr(L, name).restype = ctypes.c_int
     _lib = L
     return L
@@ -173,6 +175,16 @@ def score(h: int, coef, x, vel, scores_out, preview_out=None, stream=None) -> No
 def prune_ovf(h: int, stage: int, scores, keep_idx, src_rows=None, sel_var=None, stream=None) -> None:
     _check(lib().pg_prune_ovf(h, stage, _p(scores), _p(keep_idx), _p(src_rows), _p(sel_var),
                               _stream(stream)), "pg_prune_ovf")
+
+
+def prune_uniform(h: int, stage: int, keep_idx, src_rows=None, stream=None) -> None:
+    _check(lib().pg_prune_uniform(h, stage, _p(keep_idx), _p(src_rows), _stream(stream)), "pg_prune_uniform")
+
+
+def group_stats(n_groups: int, n: int, scores, delta: float, mean=None, std=None, clustered_frac=None,
+                stream=None) -> None:
+    _check(lib().pg_group_stats(n_groups, n, _p(scores), delta, _p(mean), _p(std), _p(clustered_frac),
+                                _stream(stream)), "pg_group_stats")
 
 
 def compact(h: int, keep_idx, src, dst, row_bytes: int, stream=None) -> None:

@@ -261,6 +261,13 @@ int launch_ovf(int n_groups, int n, int k, const float* scores, int32_t* keep_id
                int32_t* src_rows, float* sel_var, float* kept_scores, float* adv, float adv_eps,
                const int32_t* traj_in, int32_t* traj_out, int32_t* status, cudaStream_t stream);
 
+int launch_group_stats(int n_groups, int n, const float* scores, double delta, float* mean,
+                       float* std_out, float* clustered, cudaStream_t stream);
+
+int launch_uniform_select(int n_groups, int n, int k, uint64_t seed, uint32_t stage,
+                          uint32_t group_offset, int32_t* keep_idx, int32_t* src_rows,
+                          const int32_t* traj_in, int32_t* traj_out, cudaStream_t stream);
+
 int launch_advantages(int n_groups, int K, const float* rewards, float eps, float* adv,
                       float* mean, float* std_out, cudaStream_t stream);
 

@@ -539,6 +539,102 @@ int launch_advantages(int n_groups, int K, const float* rewards, float eps, floa
   return PG_OK;
 }
 
+// ---------------------------------------------------------------- diagnostics / uniform baseline
+
+// One warp per group: mean, population standard deviation and the fraction of scores inside
+// the clustered region |R - mu| <= delta * sigma (Eq. "near-mean").
+__global__ void __launch_bounds__(128)
+group_stats_kernel(int n_groups, int n, const float* scores, double delta, float* mean, float* std_out,
+                   float* clustered) {
+  const int g = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (g >= n_groups) return;
+  const float* r = scores + (size_t)g * n;
+  double s = 0.0;
+  for (int i = lane; i < n; i += 32) s += (double)r[i];
+  const double mu = warp_sum(s) / (double)n;
+  double q = 0.0;
+  for (int i = lane; i < n; i += 32) {
+    const double dlt = (double)r[i] - mu;
+    q += dlt * dlt;
+  }
+  const double sigma = sqrt(warp_sum(q) / (double)n);
+  int inside = 0;
+  for (int i = lane; i < n; i += 32) inside += (fabs((double)r[i] - mu) <= delta * sigma) ? 1 : 0;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) inside += __shfl_xor_sync(0xFFFFFFFFu, inside, o);
+  if (lane == 0) {
+    if (mean) mean[g] = (float)mu;
+    if (std_out) std_out[g] = (float)sigma;
+    if (clustered) clustered[g] = (float)((double)inside / (double)n);
+  }
+}
+
+int launch_group_stats(int n_groups, int n, const float* scores, double delta, float* mean,
+                       float* std_out, float* clustered, cudaStream_t stream) {
+  if (n_groups == 0) return PG_OK;
+  group_stats_kernel<<<(n_groups + 3) / 4, 128, 0, stream>>>(n_groups, n, scores, delta, mean, std_out,
+                                                            clustered);
+  PG_LAUNCH_CHECK();
+  return PG_OK;
+}
+
+// Uniform k-of-n subsampling per group: slot i draws the first Philox word of counter
+// (i, stage, group, stream 4); the k smallest (word, slot) pairs are kept, ascending slot order.
+__global__ void __launch_bounds__(kOvfThreads)
+uniform_select_kernel(const __grid_constant__ PhiloxKeys rk, int n, int k, uint32_t stage,
+                      uint32_t group_offset, int32_t* keep_idx, int32_t* src_rows,
+                      const int32_t* traj_in, int32_t* traj_out) {
+  __shared__ unsigned long long keys[PG_MAX_GROUP];
+  __shared__ int warp_cnt[kOvfThreads / 32];
+  const int g = blockIdx.x, tid = threadIdx.x;
+  for (int i = tid; i < n; i += kOvfThreads) {
+    const uint4 r = philox4x32_10((uint32_t)i, stage, group_offset + (uint32_t)g, 4u, rk);
+    keys[i] = ((unsigned long long)r.x << 32) | (unsigned int)i;
+  }
+  __syncthreads();
+  int running = 0;
+  for (int base = 0; base < n; base += kOvfThreads) {
+    const int i = base + tid;
+    bool keep = false;
+    if (i < n) {
+      const unsigned long long mine = keys[i];
+      int smaller = 0;
+      for (int j = 0; j < n; ++j) smaller += (keys[j] < mine) ? 1 : 0;
+      keep = smaller < k;
+    }
+    const unsigned int bal = __ballot_sync(0xFFFFFFFFu, keep);
+    if ((tid & 31) == 0) warp_cnt[tid >> 5] = __popc(bal);
+    __syncthreads();
+    int before = 0, total = 0;
+#pragma unroll
+    for (int w = 0; w < kOvfThreads / 32; ++w) {
+      const int c = warp_cnt[w];
+      if (w < (tid >> 5)) before += c;
+      total += c;
+    }
+    if (keep) {
+      const size_t o = (size_t)g * k + running + before + __popc(bal & ((1u << (tid & 31)) - 1u));
+      keep_idx[o] = i;
+      if (src_rows) src_rows[o] = g * n + i;
+      if (traj_out) traj_out[o] = traj_in[(size_t)g * n + i];
+    }
+    running += total;
+    __syncthreads();
+  }
+}
+
+int launch_uniform_select(int n_groups, int n, int k, uint64_t seed, uint32_t stage,
+                          uint32_t group_offset, int32_t* keep_idx, int32_t* src_rows,
+                          const int32_t* traj_in, int32_t* traj_out, cudaStream_t stream) {
+  if (n_groups == 0) return PG_OK;
+  uniform_select_kernel<<<n_groups, kOvfThreads, 0, stream>>>(make_philox_keys(seed), n, k, stage,
+                                                              group_offset, keep_idx, src_rows, traj_in,
+                                                              traj_out);
+  PG_LAUNCH_CHECK();
+  return PG_OK;
+}
+
 // ---------------------------------------------------------------- trajectory ids
 
 __global__ void iota_kernel(int32_t* dst, int n, int32_t base) {

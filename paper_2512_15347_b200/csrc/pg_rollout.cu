@@ -195,6 +195,32 @@ int pg_prune_ovf(pg_rollout* h, int32_t stage, const float* scores, int32_t* kee
   return PG_OK;
 }
 
+int pg_prune_uniform(pg_rollout* h, int32_t stage, int32_t* keep_idx, int32_t* src_rows, void* stream) {
+  if (!h || !keep_idx) return PG_EINVAL;
+  if (stage != h->stage_cur || stage >= h->cfg.n_stages) return PG_ESTATE;
+  if (h->stage_step[stage] != h->next_step) return PG_ESTATE;
+  const int n = h->k_cur, k = h->stage_keep[stage];
+  const int rc = pg::launch_uniform_select(h->cfg.n_groups, n, k, h->cfg.seed, (uint32_t)stage,
+                                           (uint32_t)h->cfg.group_offset, keep_idx, src_rows,
+                                           h->d_traj[h->traj_cur], h->d_traj[h->traj_cur ^ 1],
+                                           (cudaStream_t)stream);
+  if (rc != PG_OK) return rc;
+  h->traj_cur ^= 1;
+  h->k_prev = n;
+  h->k_cur = k;
+  h->stage_cur = stage + 1;
+  return PG_OK;
+}
+
+int pg_group_stats(int32_t n_groups, int32_t n, const float* scores, float delta, float* mean,
+                   float* std, float* clustered_frac, void* stream) {
+  if (n_groups < 0 || n < 1 || !(delta >= 0.f)) return PG_EINVAL;
+  if (n_groups == 0) return PG_OK;
+  if (!scores) return PG_EINVAL;
+  return pg::launch_group_stats(n_groups, n, scores, (double)delta, mean, std, clustered_frac,
+                                (cudaStream_t)stream);
+}
+
 int pg_compact(pg_rollout* h, const int32_t* keep_idx, const void* src, void* dst, size_t row_bytes,
                void* stream) {
   if (!h || !keep_idx || !src || !dst || row_bytes == 0) return PG_EINVAL;

@@ -471,3 +471,51 @@ def test_empty_batches_are_accepted(B):
     B.normal_rows(1, 0, 0, 0, 8, None, None)
     B.score_static(0, 8, B.VEL_F32, (1.0, 0.0), None, None, None)
     torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------ diagnostics and the uniform baseline
+
+def test_group_stats_match_oracle(B):
+    for G, n in [(1, 16), (64, 64), (4096, 256), (7, 1000), (3, 1)]:
+        sc = wl.clustered_scores(G, n, G + n, 0, cluster_sigma=0.05, outlier_frac=0.15,
+                                 outlier_scale=0.3, nu=3.0)
+        mean = torch.empty(G, device="cuda")
+        std = torch.empty(G, device="cuda")
+        frac = torch.empty(G, device="cuda")
+        for delta in (0.5, 1.0):
+            B.group_stats(G, n, U.to_dev(sc), delta, mean, std, frac)
+            rm, rs, rf = oracle.group_stats(sc, delta)
+            np.testing.assert_allclose(mean.cpu().numpy(), rm, rtol=1e-6, atol=1e-7)
+            np.testing.assert_allclose(std.cpu().numpy(), rs, rtol=1e-6, atol=1e-12)
+            np.testing.assert_allclose(frac.cpu().numpy(), rf, rtol=1e-6, atol=1e-7)
+
+
+def test_uniform_pruning_matches_oracle_bit_for_bit(B):
+    G, N0, d = 5, 48, 16
+    stages = [(0, 32), (1, 8), (2, 8)]
+    h, _ = _handle(B, G, N0, d, T=4, stages=stages, seed=(9 << 32) | 77, group_offset=3)
+    try:
+        x = torch.randn(G * N0, d, device="cuda")
+        lp = torch.empty(G * N0, device="cuda")
+        ids_ref = (np.arange(G * N0) + 3 * N0).astype(np.int32)
+        k_prev = N0
+        for si, (s, k) in enumerate(stages):
+            keep = torch.empty(G * k, dtype=torch.int32, device="cuda")
+            src = torch.empty(G * k, dtype=torch.int32, device="cuda")
+            B.prune_uniform(h, si, keep, src)
+            ref_keep = oracle.select_uniform(G, k_prev, k, (9 << 32) | 77, si, group_offset=3)
+            np.testing.assert_array_equal(keep.cpu().numpy().reshape(G, k), ref_keep)
+            np.testing.assert_array_equal(src.cpu().numpy(),
+                                          (ref_keep + np.arange(G)[:, None] * k_prev).reshape(-1))
+            ids_ref = oracle.compact_rows(ref_keep, ids_ref.reshape(-1, 1), k_prev).reshape(-1)
+            got_ids = torch.empty(G * k, dtype=torch.int32, device="cuda")
+            B.rollout_traj_ids(h, got_ids)
+            np.testing.assert_array_equal(got_ids.cpu().numpy(), ids_ref)
+            y = torch.empty(G * k, d, device="cuda")
+            B.step(h, s, (1.0, 0.0, 0.1), x, x, src, y, lp[: G * k])
+            x = y
+            k_prev = k
+        assert B.rollout_status(h) == (G * 8, 3, 0)
+    finally:
+        torch.cuda.synchronize()
+        B.rollout_destroy(h)
