@@ -146,6 +146,15 @@ int pg_score(pg_rollout *h, const pg_preview_coef *coef, const float *x, const v
              float *scores_out, float *preview_out, void *stream);
 
 /*
+ * Preview emission only (Eq. "ode_lookahead_method"): out[i] = p_x * x[i] + p_v * vel[i] for the
+ * n_active rows, written as fp32 (out_dtype PG_VEL_F32) or bf16 rounded to nearest even
+ * (PG_VEL_BF16), same [n_active, d] layout as the latents, for the VAE decoder and reward model
+ * of Eq. "proxy_reward_method" that run outside this library.  No reduction, no cursor change.
+ */
+int pg_preview(pg_rollout *h, const pg_preview_coef *coef, const float *x, const void *vel, void *out,
+               int32_t out_dtype, void *stream);
+
+/*
  * Optimal Variance Filtering for stage `stage` (Eq. "ovf"; Section 5.1): in
  * every group keeps the k = stage_keep[stage] of the K_i active trajectories
  * whose scores have maximal population variance.  The maximiser is found

@@ -243,6 +243,9 @@ int launch_score(int n_rows, int elems, int vel_dtype, const float* x, const voi
                  double p_x, double p_v, float* scores_out, float* preview_out,
                  RowScratch scratch, cudaStream_t stream, int forced_chunk_quads = 0);
 
+int launch_preview(int n_rows, int elems, int vel_dtype, const float* x, const void* vel, double p_x,
+                   double p_v, void* out, int out_bf16, cudaStream_t stream);
+
 int launch_policy_logprob(int n_rows, int elems, int vel_dtype, const float* x, const float* x_next,
                           const void* vel, const void* vel_ref, double c_x, double c_v,
                           double noise_std, int logp_mean, float* logp_out, float* kl_out,

@@ -178,6 +178,16 @@ int pg_score(pg_rollout* h, const pg_preview_coef* coef, const float* x, const v
                           scores_out, preview_out, scratch, (cudaStream_t)stream);
 }
 
+int pg_preview(pg_rollout* h, const pg_preview_coef* coef, const float* x, const void* vel, void* out,
+               int32_t out_dtype, void* stream) {
+  if (!h || !coef || !x || !vel || !out) return PG_EINVAL;
+  if (out_dtype != PG_VEL_F32 && out_dtype != PG_VEL_BF16) return PG_EINVAL;
+  if (!std::isfinite(coef->p_x) || !std::isfinite(coef->p_v)) return PG_EINVAL;
+  if (!aligned16(x) || !aligned16(vel) || !aligned16(out)) return PG_EINVAL;
+  return pg::launch_preview(h->cfg.n_groups * h->k_cur, h->cfg.elems, h->cfg.vel_dtype, x, vel, coef->p_x,
+                            coef->p_v, out, out_dtype == PG_VEL_BF16, (cudaStream_t)stream);
+}
+
 int pg_prune_ovf(pg_rollout* h, int32_t stage, const float* scores, int32_t* keep_idx,
                  int32_t* src_rows, float* sel_var, void* stream) {
   if (!h || !scores || !keep_idx) return PG_EINVAL;

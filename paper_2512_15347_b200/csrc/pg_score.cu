@@ -136,4 +136,74 @@ int launch_score(int n_rows, int elems, int vel_dtype, const float* x, const voi
   return PG_OK;
 }
 
+// ---------------------------------------------------------------- preview emission only
+
+__device__ __forceinline__ void store_preview(float* out, size_t quad, const float4& v) {
+  __stcs(reinterpret_cast<float4*>(out) + quad, v);
+}
+__device__ __forceinline__ void store_preview(__nv_bfloat16* out, size_t quad, const float4& v) {
+  const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
+  const __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 w;
+  w.x = *reinterpret_cast<const unsigned int*>(&lo);
+  w.y = *reinterpret_cast<const unsigned int*>(&hi);
+  __stcs(reinterpret_cast<uint2*>(out) + quad, w);
+}
+
+// x_hat = p_x x + p_v v written in fp32 or bf16 (for a decoder that follows); no reduction.
+template <typename VelT, typename OutT>
+__global__ void __launch_bounds__(kRowThreads)
+preview_kernel(const float* __restrict__ x, const void* __restrict__ vel_v, OutT* __restrict__ out,
+               long long total_quads, float p_x, float p_v) {
+  using Raw = typename VelRaw<VelT>::type;
+  const Raw* vel = reinterpret_cast<const Raw*>(vel_v);
+  constexpr int kU = 4;
+  const long long stride = (long long)gridDim.x * kRowThreads * kU;
+  for (long long q0 = (long long)blockIdx.x * kRowThreads * kU + threadIdx.x; q0 < total_quads; q0 += stride) {
+    float4 xv[kU];
+    Raw vv[kU];
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      const long long q = q0 + u * kRowThreads;
+      if (q < total_quads) {
+        xv[u] = __ldcs(reinterpret_cast<const float4*>(x) + q);
+        vv[u] = __ldcs(vel + q);
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kU; ++u) {
+      const long long q = q0 + u * kRowThreads;
+      if (q < total_quads) {
+        const float4 vf = unpack_vel(vv[u]);
+        float4 h;
+        h.x = fmaf(p_v, vf.x, p_x * xv[u].x);
+        h.y = fmaf(p_v, vf.y, p_x * xv[u].y);
+        h.z = fmaf(p_v, vf.z, p_x * xv[u].z);
+        h.w = fmaf(p_v, vf.w, p_x * xv[u].w);
+        store_preview(out, (size_t)q, h);
+      }
+    }
+  }
+}
+
+int launch_preview(int n_rows, int elems, int vel_dtype, const float* x, const void* vel, double p_x,
+                   double p_v, void* out, int out_bf16, cudaStream_t stream) {
+  const long long total = (long long)n_rows * (elems / 4);
+  if (total == 0) return PG_OK;
+  const long long per_cta = (long long)kRowThreads * 4 * 4;          // 16 quads per thread
+  long long ctas = (total + per_cta - 1) / per_cta;
+  if (ctas > 148LL * 64) ctas = 148LL * 64;
+  const dim3 grid((unsigned)ctas), block(kRowThreads);
+  const float px = (float)p_x, pv = (float)p_v;
+  if (vel_dtype == PG_VEL_BF16) {
+    if (out_bf16) preview_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, block, 0, stream>>>(x, vel, (__nv_bfloat16*)out, total, px, pv);
+    else          preview_kernel<__nv_bfloat16, float><<<grid, block, 0, stream>>>(x, vel, (float*)out, total, px, pv);
+  } else {
+    if (out_bf16) preview_kernel<float, __nv_bfloat16><<<grid, block, 0, stream>>>(x, vel, (__nv_bfloat16*)out, total, px, pv);
+    else          preview_kernel<float, float><<<grid, block, 0, stream>>>(x, vel, (float*)out, total, px, pv);
+  }
+  PG_LAUNCH_CHECK();
+  return PG_OK;
+}
+
 }  // namespace pg

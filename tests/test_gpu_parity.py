@@ -519,3 +519,65 @@ def test_uniform_pruning_matches_oracle_bit_for_bit(B):
     finally:
         torch.cuda.synchronize()
         B.rollout_destroy(h)
+
+
+def test_host_buffer_rollout_with_external_scores_and_rewards(B):
+    """pg_rollout_host fed with reward-model style inputs: per-stage scores and final rewards from
+    the host instead of the preview mean."""
+    w = wl.scaled(wl.WORKLOADS["sd3"], n_groups=3, elems=4096 + 64)
+    inp = U.SharedInputs(w)
+    ref = U.run_oracle(w, inp)
+    cfg = B.make_config(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, B.VEL_BF16,
+                        adv_eps=w.adv_eps)
+    ws = torch.empty(B.rollout_host_workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+    x0 = torch.from_numpy(inp.x0).pin_memory()
+    vels = [U.vel_to_dev(inp.vel_numpy(s, np.empty((w.n_groups * w.rows_before(s), 0)))).cpu().pin_memory()
+            for s in range(w.n_steps)]
+    # the stand-in reward model is keyed by original trajectory: replay the oracle's survivors
+    stage_ids = [np.arange(w.n_groups * w.n_expand, dtype=np.int32)]
+    for keep, (s, k) in zip(ref.stage_keep, w.stages):
+        prev = stage_ids[-1].reshape(w.n_groups, -1)
+        stage_ids.append(np.take_along_axis(prev, keep, axis=1).reshape(-1))
+    stage_scores = [torch.from_numpy(wl.sd3_stage_scores(w, i, stage_ids[i])).pin_memory()
+                    for i in range(len(w.stages))]
+    final = torch.from_numpy(wl.sd3_stage_scores(w, 99, stage_ids[-1])).pin_memory()
+    K = w.final_keep
+    x_final = torch.empty(w.n_groups * K, w.elems).pin_memory()
+    logp = torch.empty(w.traj_steps).pin_memory()
+    keep = torch.empty(sum(w.n_groups * k for _, k in w.stages), dtype=torch.int32).pin_memory()
+    adv = torch.empty(w.n_groups * K).pin_memory()
+    ids = torch.empty(w.n_groups * K, dtype=torch.int32).pin_memory()
+    rc = B.rollout_host(cfg, [w.step_coef(s) for s in range(w.n_steps)], [], x0, vels, stage_scores,
+                        final, x_final, logp, keep, adv, ids, ws)
+    assert rc == 0
+    np.testing.assert_array_equal(keep.numpy(), np.concatenate([k.reshape(-1) for k in ref.stage_keep]))
+    np.testing.assert_array_equal(ids.numpy(), ref.traj_id)
+    assert U.latent_err(x_final.numpy(), ref.x_final) <= U.LATENT_TOL
+    assert U.logp_err(logp.numpy(), np.concatenate(ref.logp), w.elems) <= U.LOGP_TOL
+    np.testing.assert_allclose(adv.numpy().reshape(w.n_groups, K), ref.adv, rtol=1e-5, atol=1e-6)
+
+
+@pytest.mark.parametrize("bf16_vel", [False, True])
+@pytest.mark.parametrize("d", [4, 3 * 8192 + 20])
+def test_preview_emission_matches_oracle(B, bf16_vel, d):
+    n_groups, n0 = 2, 5
+    n = n_groups * n0
+    rng = np.random.default_rng(d)
+    x = rng.standard_normal((n, d)).astype(np.float32)
+    vt = torch.from_numpy(rng.standard_normal((n, d)).astype(np.float32))
+    vt = vt.to(torch.bfloat16) if bf16_vel else vt
+    v = wl.as_numpy_velocity(vt)
+    h, _ = _handle(B, n_groups, n0, d, bf16=bf16_vel)
+    try:
+        _, ref = oracle.score(x, v, 0.9, 0.4, want_preview=True)
+        out32 = torch.empty(n, d, device="cuda")
+        out16 = torch.empty(n, d, device="cuda", dtype=torch.bfloat16)
+        B.preview(h, (0.9, 0.4), U.to_dev(x), U.vel_to_dev(v), out32)
+        B.preview(h, (0.9, 0.4), U.to_dev(x), U.vel_to_dev(v), out16)
+        assert U.latent_err(out32.cpu().numpy(), ref) <= 1e-6
+        # bf16: 8 significant bits, round to nearest
+        assert U.latent_err(out16.float().cpu().numpy(), ref) <= 2.0 ** -8
+        assert torch.equal(out16, out32.to(torch.bfloat16))
+    finally:
+        torch.cuda.synchronize()
+        B.rollout_destroy(h)
