@@ -31,3 +31,15 @@ def max_over_ranks(value: float, dist=None, device=None) -> float:
     t = torch.tensor([value], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def all_gather_groups(t, dist=None):
+    """Concatenates a per-group (or per-trajectory) tensor over ranks in rank order, i.e. in global
+    group order for contiguous shards of equal size.  The only collective the sharded rollout can
+    need: a few KB of advantages / statistics when one rank wants the whole batch."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return t
+    import torch
+    parts = [torch.empty_like(t) for _ in range(dist.get_world_size())]
+    dist.all_gather(parts, t.contiguous())
+    return torch.cat(parts, dim=0)

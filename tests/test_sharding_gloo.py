@@ -38,6 +38,11 @@ def _worker(rank, world, port, total_groups, out_dir):
         # timing reduction: every rank must see the slowest rank's time
         slowest = sharding.max_over_ranks(10.0 + rank, dist)
         assert slowest == 10.0 + world - 1
+        # equal shards gather back into global group order
+        mine = torch.full((2, 3), float(rank))
+        whole = sharding.all_gather_groups(mine, dist)
+        assert whole.shape == (2 * world, 3)
+        assert torch.equal(whole[:, 0], torch.arange(world).repeat_interleave(2).float())
         dist.barrier()
     finally:
         dist.destroy_process_group()
