@@ -30,7 +30,7 @@ if ROOT not in sys.path:
 
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) over algorithmic bytes of the step
 # kernel, from the ncu capture summarised in profiles/step_kernel_bf16_1024rows.txt (1024-row
-# launch: 2.642 GB measured, 2.684 GB algorithmic).  Set to None whenever the kernel changes
+# launch: 2.640 GB measured, 2.684 GB algorithmic).  Set to None whenever the kernel changes
 # until the counters are taken again.
 STEP_KERNEL_TRAFFIC_RATIO = 0.984
 

@@ -64,35 +64,40 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
   return make_uint4(c0, c1, c2, c3);
 }
 
-// Two standard normals from two generator words (24-bit uniforms, Box-Muller).
+// Box-Muller on two generator words (24-bit uniforms):
 //   u1 = ((r0 >> 8) + 1) * 2^-24 in (0, 1],  u2 = (r1 >> 8) * 2^-24 in [0, 1)
-//   a = sqrt(-2 ln u1) cos(2 pi u2),  b = sqrt(-2 ln u1) sin(2 pi u2)
-// Returns -2 ln u1 = a^2 + b^2 (the pair's contribution to the sum of squared noise).
+//   normals  a = sqrt(-2 ln u1) cos(2 pi u2),  b = sqrt(-2 ln u1) sin(2 pi u2)
+// Returned in factored form: radius = sqrt(-2 ln u1) and (c, s) = (cos, sin)(2 pi u2 - pi), so
+// that a = -radius * c and b = -radius * s (half-turn shift: the hardware sine / cosine are
+// evaluated on [-pi, pi), their most accurate range); the return value is -2 ln u1 = a^2 + b^2.
 // The logarithm uses the hardware log2 except close to u1 = 1, where its absolute error would
 // dominate the small radius: there -2 ln(1 - w) is summed as a short series in w = 1 - u1 (exact
-// in fp32; truncation below 2e-8 relative for w < 2^-6).  The angle is shifted by half a turn
-// (cos(t) = -cos(t - pi), same for sin) so that the hardware sine / cosine are evaluated on
-// [-pi, pi), their most accurate range.
-__device__ __forceinline__ float normal_pair(uint32_t r0, uint32_t r1, float& a, float& b) {
+// in fp32; truncation below 2e-8 relative for w < 2^-6).
+__device__ __forceinline__ float box_muller(uint32_t r0, uint32_t r1, float& radius, float& c, float& s) {
   const float k1 = (float)(r0 >> 8);
   const float u1 = fmaf(k1, 5.9604644775390625e-8f, 5.9604644775390625e-8f);
   float lg;                                                     // u1 >= 2^-24: never subnormal
   asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(u1));
   float neg2ln = -1.3862943611198906f * lg;                     // -2 ln(u1) = -2 ln2 * log2(u1)
-  const float w = 1.0f - u1;                                     // exact (Sterbenz / 24-bit grid)
+  const float w = 1.0f - u1;                                     // exact (24-bit grid)
   // -2 ln(1 - w) = 2w + w^2 + (2/3) w^3 + (1/2) w^4 + ...
   float ser = fmaf(w, 0.5f, 0.66666666666666667f);
   ser = fmaf(ser, w, 1.0f);
   ser = fmaf(ser, w, 2.0f);
   ser *= w;
   neg2ln = (w < 0.015625f) ? ser : neg2ln;
-  float radius;
   asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(radius) : "f"(neg2ln));
   const float turn = fmaf((float)(r1 >> 8), 5.9604644775390625e-8f, -0.5f);  // u2 - 1/2, exact
   const float angle = 6.283185307179586f * turn;
-  float s, c;
   asm("sin.approx.ftz.f32 %0, %1;" : "=f"(s) : "f"(angle));
   asm("cos.approx.ftz.f32 %0, %1;" : "=f"(c) : "f"(angle));
+  return neg2ln;
+}
+
+// The two normals themselves.
+__device__ __forceinline__ float normal_pair(uint32_t r0, uint32_t r1, float& a, float& b) {
+  float radius, c, s;
+  const float neg2ln = box_muller(r0, r1, radius, c, s);
   a = -radius * c;
   b = -radius * s;
   return neg2ln;

@@ -2,7 +2,8 @@
 //
 // One CTA streams one chunk of one trajectory: x and the prediction are read once with
 // 128/64-bit coalesced loads (the loads of the next pair of quads are issued before the
-// current pair is computed), the noise is generated in registers (one Philox block per 4
+// current pair is computed; full chunks alternate between two register sets without bounds
+// checks), the noise is generated in registers (one Philox block per 4
 // elements), x' is written once.  Sum of squared noise: for a Box-Muller pair a^2 + b^2 equals
 // -2 ln u1, so the radius term is accumulated directly.  The per-trajectory sum is reduced
 // thread -> warp (shuffle) -> trajectory (fixed-slot partials finished by the last-arriving
@@ -24,7 +25,7 @@ struct StepParams {
   int chunk_quads;        // quads per CTA
   int chunks;             // CTAs per row
   uint32_t step;
-  float c_x, c_v, noise_std;
+  float c_x, c_v, neg_noise_std;
   double logp_const;      // d/2 * ln(2 pi noise_std^2)
   double logp_scale;      // 1 or 1/d
   PhiloxKeys rk;
@@ -59,6 +60,8 @@ template <> struct VelReg<__nv_bfloat16> { using type = VelBf16; };
 #define PG_STEP_MIN_CTAS 5     // __launch_bounds__ minimum resident CTAs per SM
 #endif
 constexpr int kStepUnroll = PG_STEP_UNROLL;
+static_assert(kMinChunkQuads % (2 * kStepUnroll * kRowThreads) == 0 && kMaxChunkQuads % kMinChunkQuads == 0,
+              "full chunks must hold an even number of batches");
 
 // One quad: mean of the transition, noise, store, radius-term accumulation.
 template <bool kNoise, bool kUnitCx>
@@ -78,13 +81,16 @@ __device__ __forceinline__ void step_quad(const StepParams& p, uint32_t traj, in
   }
   if (kNoise) {
     const uint4 r = philox4x32_10((uint32_t)q, p.step, traj, 0u, p.rk);
-    float n0, n1, n2, n3;
-    acc += normal_pair(r.x, r.y, n0, n1);
-    acc += normal_pair(r.z, r.w, n2, n3);
-    m.x = fmaf(p.noise_std, n0, m.x);
-    m.y = fmaf(p.noise_std, n1, m.y);
-    m.z = fmaf(p.noise_std, n2, m.z);
-    m.w = fmaf(p.noise_std, n3, m.w);
+    // noise_std * xi = (-noise_std * radius) * (cos, sin): the scale is applied once per pair
+    float ra, ca, sa, rb, cb, sb;
+    acc += box_muller(r.x, r.y, ra, ca, sa);
+    acc += box_muller(r.z, r.w, rb, cb, sb);
+    ra *= p.neg_noise_std;
+    rb *= p.neg_noise_std;
+    m.x = fmaf(ra, ca, m.x);
+    m.y = fmaf(ra, sa, m.y);
+    m.z = fmaf(rb, cb, m.z);
+    m.w = fmaf(rb, sb, m.w);
   }
   __stcs(xout + q, m);
 }
@@ -109,11 +115,46 @@ step_kernel(const __grid_constant__ StepParams p) {
   float4 xv[kStepUnroll], nx[kStepUnroll];
   VReg vv[kStepUnroll], nv[kStepUnroll];
   int q = q_begin + threadIdx.x;
+  if (q_end - q_begin == p.chunk_quads) {
+    // full chunk (a multiple of 2 * kStepUnroll * kRowThreads quads): two register sets take
+    // turns, no bounds checks and no register copies
+    constexpr int kStride = kStepUnroll * kRowThreads;
+    const int iters = p.chunk_quads / kStride;          // even
 #pragma unroll
-  for (int u = 0; u < kStepUnroll; ++u) {
-    const int qq = q + u * kRowThreads;
-    if (qq < q_end) { xv[u] = __ldcs(xin + qq); load_vel(vel, (size_t)qq, vv[u]); }
+    for (int u = 0; u < kStepUnroll; ++u) {
+      xv[u] = __ldcs(xin + q + u * kRowThreads);
+      load_vel(vel, (size_t)(q + u * kRowThreads), vv[u]);
+    }
+    for (int it = 0; it < iters; it += 2) {
+#pragma unroll
+      for (int u = 0; u < kStepUnroll; ++u) {
+        nx[u] = __ldcs(xin + q + kStride + u * kRowThreads);
+        load_vel(vel, (size_t)(q + kStride + u * kRowThreads), nv[u]);
+      }
+#pragma unroll
+      for (int u = 0; u < kStepUnroll; ++u)
+        step_quad<kNoise, kUnitCx>(p, traj, q + u * kRowThreads, xv[u], vel_f32(vv[u]), xout, acc);
+      if (it + 2 < iters) {
+#pragma unroll
+        for (int u = 0; u < kStepUnroll; ++u) {
+          xv[u] = __ldcs(xin + q + 2 * kStride + u * kRowThreads);
+          load_vel(vel, (size_t)(q + 2 * kStride + u * kRowThreads), vv[u]);
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < kStepUnroll; ++u)
+        step_quad<kNoise, kUnitCx>(p, traj, q + kStride + u * kRowThreads, nx[u], vel_f32(nv[u]), xout, acc);
+      q += 2 * kStride;
+    }
+    q = q_end;
+  } else {
+#pragma unroll
+    for (int u = 0; u < kStepUnroll; ++u) {
+      const int qq = q + u * kRowThreads;
+      if (qq < q_end) { xv[u] = __ldcs(xin + qq); load_vel(vel, (size_t)qq, vv[u]); }
+    }
   }
+  // ragged last chunk of a row: guarded loop
   while (q < q_end) {
     const int nq = q + kStepUnroll * kRowThreads;
 #pragma unroll
@@ -174,7 +215,7 @@ int launch_step(int n_rows, int elems, int vel_dtype, const float* x_in, const v
   p.step = (uint32_t)step;
   p.c_x = (float)c_x;
   p.c_v = (float)c_v;
-  p.noise_std = (float)noise_std;
+  p.neg_noise_std = -(float)noise_std;
   const double two_pi = 6.283185307179586476925286766559;
   p.logp_const = noise_std > 0.0 ? 0.5 * (double)elems * log(two_pi * noise_std * noise_std) : 0.0;
   p.logp_scale = logp_mean ? 1.0 / (double)elems : 1.0;
