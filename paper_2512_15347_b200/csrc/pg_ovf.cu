@@ -27,6 +27,7 @@ struct OvfParams {
   int32_t* status;          // device word or null
   int n, k;
   float adv_eps;
+  int bulk_ok;              // scores base is 16-byte aligned: rows may be staged with a bulk copy
 };
 
 // Monotone map fp32 -> uint32: a < b (as floats, -0 == +0, NaN highest) <=> key(a) < key(b).
@@ -246,7 +247,11 @@ ovf_select_kernel(const __grid_constant__ OvfParams p) {
 
 // ---------------------------------------------------------------- groups of up to 256 scores
 //
-// One warp per group, E = 1, 2, 4 or 8 scores per lane (n <= 32 * E), no CTA barrier.
+// One warp per group, E = 1, 2, 4 or 8 scores per lane (n <= 32 * E); the four warps of a CTA
+// only meet once, for the staging of their score rows.
+//  0. The CTA's score rows are staged in shared memory by one bulk asynchronous copy
+//     (cp.async.bulk, completion on an mbarrier, bounded wait) when source and size are
+//     16-byte aligned, else read with ordinary loads.
 //  1. The 32-bit order keys alone are sorted with a bitonic network held in registers (one
 //     integer min and one max per compare-exchange; shuffles for distances of E and more).
 //     Slots >= n hold an all-ones key and sort to the end.
@@ -259,6 +264,7 @@ ovf_select_kernel(const __grid_constant__ OvfParams p) {
 //  4. k+1 candidates, argmax with the "largest j" tie rule, membership by rank; every lane holds
 //     its scores in slot order, so a popcount prefix over lanes gives ascending slot order.
 constexpr int kOvfWarpsPerCta = 4;
+constexpr int kBulkWaitLimit = 1 << 14;   // mbarrier try_wait attempts before giving up
 
 __device__ __forceinline__ float key_to_score(uint32_t key) {
   const uint32_t b = (key & 0x80000000u) ? (key ^ 0x80000000u) : ~key;
@@ -270,12 +276,55 @@ __global__ void __launch_bounds__(kOvfWarpsPerCta * 32)
 ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
   constexpr int N = 32 * E;
   extern __shared__ __align__(16) unsigned char smem[];
+  __shared__ __align__(8) unsigned long long stage_bar;
   const int n = p.n, k = p.k;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g = blockIdx.x * kOvfWarpsPerCta + warp;
+  const int g0 = blockIdx.x * kOvfWarpsPerCta;
+  const int g = g0 + warp;
+
+  // 0. stage the score rows of this CTA's groups (contiguous in memory) in shared memory with
+  //    one bulk asynchronous copy, completion signalled on an mbarrier.  Needs a 16-byte
+  //    aligned source and size; otherwise the rows are read with ordinary loads.  The wait is
+  //    bounded: if the copy has not landed in time, status bit 1 is set and the CTA gives up.
+  float* stage = reinterpret_cast<float*>(smem);                 // [kOvfWarpsPerCta * n]
+  const int groups_here = min(kOvfWarpsPerCta, n_groups - g0);
+  const unsigned int stage_bytes = (unsigned int)groups_here * (unsigned int)n * 4u;
+  const bool bulk = p.bulk_ok && (stage_bytes & 15u) == 0 && ((((size_t)g0 * n * 4) & 15) == 0);
+  if (bulk) {                                                    // uniform over the CTA
+    const unsigned int bar = (unsigned int)__cvta_generic_to_shared(&stage_bar);
+    const unsigned int dst = (unsigned int)__cvta_generic_to_shared(stage);
+    if (threadIdx.x == 0) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      const float* src = p.scores + (size_t)g0 * n;
+      asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(stage_bytes)
+                   : "memory");
+      asm volatile(
+          "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+          "l"(src), "r"(stage_bytes), "r"(bar)
+          : "memory");
+    }
+    unsigned int done = 0;
+    for (int round = 0; round < 2 && !done; ++round) {
+      for (int it = 0; it < kBulkWaitLimit && !done; ++it) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done)
+            : "r"(bar), "r"(0u)
+            : "memory");
+      }
+      if (!done && round == 0 && threadIdx.x == 0 && p.status) atomicOr(p.status, 2);
+    }
+    if (!done) return;        // waited twice without success: leave, the host reads the status
+  }
   if (g >= n_groups) return;
   const size_t per_warp = (size_t)(k + 1) * 4 * sizeof(double) + (size_t)N * 2 * sizeof(uint32_t);
-  unsigned char* base = smem + (size_t)warp * per_warp;
+  unsigned char* base = smem + (size_t)kOvfWarpsPerCta * N * sizeof(float) + (size_t)warp * per_warp;
   double* L1 = reinterpret_cast<double*>(base);
   double* L2 = L1 + (k + 1);
   double* H1 = L2 + (k + 1);
@@ -291,7 +340,7 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
   for (int r = 0; r < E; ++r) {
     const int i = lane * E + r;
     if (i < n) {
-      orig[r] = sc[i];
+      orig[r] = bulk ? stage[warp * n + i] : sc[i];
       bad |= !(fabsf(orig[r]) <= FLT_MAX);
       mine[r] = order_key(orig[r]);
     } else {
@@ -469,8 +518,9 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
 template <int E>
 static void launch_ovf_warp(const OvfParams& p, int n_groups, cudaStream_t stream) {
   const size_t per_warp = (size_t)(p.k + 1) * 4 * sizeof(double) + (size_t)(32 * E) * 2 * sizeof(uint32_t);
+  const size_t stage = (size_t)kOvfWarpsPerCta * 32 * E * sizeof(float);
   const int ctas = (n_groups + kOvfWarpsPerCta - 1) / kOvfWarpsPerCta;
-  ovf_warp_kernel<E><<<ctas, kOvfWarpsPerCta * 32, per_warp * kOvfWarpsPerCta, stream>>>(p, n_groups);
+  ovf_warp_kernel<E><<<ctas, kOvfWarpsPerCta * 32, stage + per_warp * kOvfWarpsPerCta, stream>>>(p, n_groups);
 }
 
 int launch_ovf(int n_groups, int n, int k, const float* scores, int32_t* keep_idx,
@@ -490,6 +540,7 @@ int launch_ovf(int n_groups, int n, int k, const float* scores, int32_t* keep_id
   p.n = n;
   p.k = k;
   p.adv_eps = adv_eps;
+  p.bulk_ok = (((uintptr_t)scores) & 15) == 0;
   if (n <= 32)       launch_ovf_warp<1>(p, n_groups, stream);
   else if (n <= 64)  launch_ovf_warp<2>(p, n_groups, stream);
   else if (n <= 128) launch_ovf_warp<4>(p, n_groups, stream);

@@ -581,3 +581,19 @@ def test_preview_emission_matches_oracle(B, bf16_vel, d):
     finally:
         torch.cuda.synchronize()
         B.rollout_destroy(h)
+
+
+def test_ovf_misaligned_and_ragged_score_rows(B):
+    """Score rows that cannot be staged with a bulk copy (base not 16-byte aligned, or a CTA's rows
+    not a multiple of 16 bytes) take the ordinary-load path and give the same selection."""
+    rng = np.random.default_rng(5)
+    for G, n, k in [(9, 25, 7), (6, 256, 32), (5, 3, 2), (4, 64, 16), (7, 31, 31)]:
+        sc = rng.standard_normal((G, n)).astype(np.float32)
+        ref_keep, _ = oracle.ovf_select(sc, k)
+        for shift in (0, 1, 2):
+            buf = torch.zeros(G * n + 4, device="cuda")
+            view = buf[shift: shift + G * n]
+            view.copy_(torch.from_numpy(sc).reshape(-1))
+            keep = torch.empty(G * k, dtype=torch.int32, device="cuda")
+            B.ovf_select_batched(G, n, k, view, keep)
+            np.testing.assert_array_equal(keep.cpu().numpy().reshape(G, k), ref_keep)
