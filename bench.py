@@ -317,6 +317,34 @@ def run_ours(args):
                "workload": f"{m['n_groups']} groups x {m['n']} scores -> {m['k']} (select + index/score "
                            "compaction + advantages), L2 flushed between repetitions"}
 
+    # the same rollout through the one-call native driver and as a replayed CUDA graph
+    drivers = None
+    if rank == 0 and w.velocity == "normal" and w.scores == "preview":
+        from paper_2512_15347_b200.rollout import NativeRollout
+        nat = NativeRollout(ro, [w.step_coef(s) for s in range(w.n_steps)],
+                            [w.preview_coef(s) for s, _ in w.stages], vels)
+
+        def time_calls(fn, reps):
+            fn()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(reps):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps
+        reps = max(5, min(args.steps, 50))
+        native_ms = time_calls(lambda: nat.run(x0), reps)
+        nat.capture(x0)
+        graph_ms = time_calls(lambda: nat.graph.replay(), reps)
+        drivers = {"stepwise_ms_per_rollout": total_ms / args.steps, "native_ms_per_rollout": native_ms,
+                   "graph_ms_per_rollout": graph_ms,
+                   "graph_latent_steps_per_s": w.traj_steps / (graph_ms * 1e-3),
+                   "note": "stepwise = one library call per kernel from Python (the timed `value`); native = "
+                           "pg_rollout_run, one call per rollout; graph = that call captured and replayed"}
+        del nat
+
     # policy-update kernels on the survivors' shape (secondary numbers; not part of `value`)
     policy = None
     if rank == 0 and w.vel_dtype == "bf16" and w.velocity == "normal":
@@ -375,7 +403,7 @@ def run_ours(args):
                                 v["launches"] // args.steps} for k, v in kinds.items()},
                 "score_gbs": score_gbs, "prune_stage_gbs": prune_stage_gbs,
                 "hbm_gbs_whole_rollout": (step_bytes + (score_bytes if score_gbs else 0)) / (total_ms * 1e-3) / 1e9,
-                "ovf_microbench": ovf, "policy_update": policy, "e2e": e2e, "cpu_baseline": cpu_base}
+                "ovf_microbench": ovf, "drivers": drivers, "policy_update": policy, "e2e": e2e, "cpu_baseline": cpu_base}
         print(json.dumps(line))
     ro.close()
     if dist is not None:

@@ -318,6 +318,35 @@ int pg_rollout_host(const pg_config *cfg, const pg_step_coef *step_coef,
 int pg_score_static(int32_t n_rows, int32_t elems, int32_t vel_dtype, const pg_preview_coef *coef,
                     const float *x, const void *vel, float *scores_out, void *stream);
 
+/*
+ * Whole rollout from DEVICE buffers on an existing handle (Section 5.1 + 5.2 end to end): resets
+ * the handle, then enqueues score / OVF / step for every step and the final reward stand-in and
+ * advantages, all on `stream`, without synchronising and without allocating - the sequence of
+ * launches is fixed by the schedule, so a caller may capture the call in a CUDA graph and replay
+ * it (the usual remedy when the latents are small and the rollout is launch-bound).
+ *   x0 device [G*N0, d] fp32 (only read); vel_steps HOST array of T device pointers, vel_steps[s]
+ *   being [rows_s, d] in cfg.vel_dtype (rows_s as for pg_rollout_host); stage_scores NULL or a
+ *   HOST array of I device pointers (NULL entry = preview mean); final_rewards device or NULL.
+ *   workspace: device memory of at least pg_rollout_run_workspace_bytes(cfg) bytes, 16-byte
+ *   aligned; results live inside it and are described by *out (device pointers; logp packed step
+ *   after step, keep_idx stage after stage).
+ */
+typedef struct {
+  const float *x_final;      /* [n_final, d]          */
+  const float *logp;         /* [n_logp]              */
+  const int32_t *keep_idx;   /* [n_keep]              */
+  const float *adv;          /* [n_final]             */
+  const float *rewards;      /* [n_final]             */
+  const int32_t *traj_id;    /* [n_final]             */
+  int32_t n_final;
+  int64_t n_logp, n_keep;
+} pg_rollout_outputs;
+size_t pg_rollout_run_workspace_bytes(const pg_config *cfg);
+int pg_rollout_run(pg_rollout *h, const pg_step_coef *step_coef, const pg_preview_coef *preview_coef,
+                   const float *x0, const void *const *vel_steps, const float *const *stage_scores,
+                   const float *final_rewards, void *workspace, size_t workspace_bytes,
+                   pg_rollout_outputs *out, void *stream);
+
 /* Copies the handle's current trajectory-id map ([n_active] int32, device
  * memory) to `dst` (device) in stream order. */
 int pg_rollout_traj_ids(pg_rollout *h, int32_t *dst, void *stream);

@@ -43,6 +43,12 @@ class StepCoef(ctypes.Structure):
     _fields_ = [("c_x", ctypes.c_double), ("c_v", ctypes.c_double), ("noise_std", ctypes.c_double)]
 
 
+class RolloutOutputs(ctypes.Structure):
+    _fields_ = [("x_final", ctypes.c_void_p), ("logp", ctypes.c_void_p), ("keep_idx", ctypes.c_void_p),
+                ("adv", ctypes.c_void_p), ("rewards", ctypes.c_void_p), ("traj_id", ctypes.c_void_p),
+                ("n_final", ctypes.c_int32), ("n_logp", ctypes.c_int64), ("n_keep", ctypes.c_int64)]
+
+
 class PreviewCoef(ctypes.Structure):
     _fields_ = [("p_x", ctypes.c_double), ("p_v", ctypes.c_double)]
 
@@ -83,6 +89,11 @@ def lib() -> ctypes.CDLL:
                                   ctypes.POINTER(PreviewCoef), vp, ctypes.POINTER(vp),
                                   ctypes.POINTER(vp), vp, vp, vp, vp, vp, vp, vp, sz]
     L.pg_score_static.argtypes = [i32, i32, i32, ctypes.POINTER(PreviewCoef), vp, vp, vp, vp]
+    L.pg_rollout_run_workspace_bytes.argtypes = [ctypes.POINTER(Config)]
+    L.pg_rollout_run_workspace_bytes.restype = sz
+    L.pg_rollout_run.argtypes = [vp, ctypes.POINTER(StepCoef), ctypes.POINTER(PreviewCoef), vp,
+                                 ctypes.POINTER(vp), ctypes.POINTER(vp), vp, vp, sz,
+                                 ctypes.POINTER(RolloutOutputs), vp]
     L.pg_rollout_traj_ids.argtypes = [vp, vp, vp]
     L.pg_philox_raw.argtypes = [i64, vp, vp, vp, vp]
     L.pg_normal_rows.argtypes = [u64, i32, i32, i32, i32, vp, vp, vp]
@@ -94,7 +105,7 @@ def lib() -> ctypes.CDLL:
                  "pg_step", "pg_score", "pg_prune_ovf", "pg_compact", "pg_advantages",
                  "pg_ovf_select_batched", "pg_rollout_host", "pg_rollout_traj_ids",
                  "pg_philox_raw", "pg_normal_rows", "pg_score_static", "pg_policy_logprob",
-                 "pg_policy_objective", "pg_policy_backward", "pg_prune_uniform", "pg_group_stats", "pg_preview"):
+                 "pg_policy_objective", "pg_policy_backward", "pg_prune_uniform", "pg_group_stats", "pg_preview", "pg_rollout_run"):
         getattr(L, name).restype = ctypes.c_int
     _lib = L
     return L
@@ -274,6 +285,32 @@ def rollout_host(cfg: Config, step_coefs, preview_coefs, x0, vel_steps, stage_sc
     if rc not in (OK, ENONFINITE):
         raise PgError(rc, "pg_rollout_host")
     return rc
+
+
+def rollout_run_workspace_bytes(cfg: Config) -> int:
+    return int(lib().pg_rollout_run_workspace_bytes(ctypes.byref(cfg)))
+
+
+class RunArgs:
+    """Marshalled arguments of pg_rollout_run, built once and reusable (e.g. under graph capture)."""
+
+    def __init__(self, step_coefs, preview_coefs, vel_steps, stage_scores=None):
+        self.sc = (StepCoef * len(step_coefs))(*[StepCoef(*c) for c in step_coefs])
+        self.pc = (PreviewCoef * max(len(preview_coefs), 1))(*[PreviewCoef(*c) for c in preview_coefs])
+        self.vs = (ctypes.c_void_p * len(vel_steps))(*[_p(v) for v in vel_steps])
+        self.ss = None
+        if stage_scores is not None:
+            self.ss = (ctypes.c_void_p * max(len(stage_scores), 1))(*[_p(t) for t in stage_scores])
+        self.keep = (vel_steps, stage_scores)
+        self.out = RolloutOutputs()
+
+
+def rollout_run(h: int, args: "RunArgs", x0, final_rewards, workspace, stream=None) -> RolloutOutputs:
+    """pg_rollout_run: the whole schedule from device tensors, enqueued on one stream."""
+    _check(lib().pg_rollout_run(h, args.sc, args.pc, _p(x0), args.vs, args.ss, _p(final_rewards),
+                                _p(workspace), workspace.numel() * workspace.element_size(),
+                                ctypes.byref(args.out), _stream(stream)), "pg_rollout_run")
+    return args.out
 
 
 def strerror(code: int) -> str:

@@ -502,4 +502,113 @@ int pg_rollout_host(const pg_config* cfg, const pg_step_coef* step_coef,
 #undef PG_TRY_CUDA
 }
 
+// ---------------------------------------------------------------- device-resident driver
+
+struct RunPlan {
+  size_t rows0, x_bytes, total_logp, total_keep;
+  size_t off_x[2], off_scores, off_keep, off_src, off_logp, off_rewards, off_adv, off_traj, total;
+};
+
+static RunPlan make_run_plan(const pg_config* c) {
+  RunPlan p;
+  const HostPlan hp = make_plan(c);
+  p.rows0 = hp.rows0;
+  p.x_bytes = hp.x_bytes;
+  p.total_logp = hp.total_logp;
+  p.total_keep = hp.total_keep;
+  size_t o = 0;
+  for (int i = 0; i < 2; ++i) { p.off_x[i] = o; o += round256(p.x_bytes); }
+  p.off_scores = o;  o += round256(p.rows0 * 4);
+  p.off_keep = o;    o += round256((p.total_keep + 1) * 4);
+  p.off_src = o;     o += round256(p.rows0 * 4);
+  p.off_logp = o;    o += round256(p.total_logp * 4);
+  p.off_rewards = o; o += round256(p.rows0 * 4);
+  p.off_adv = o;     o += round256(p.rows0 * 4);
+  p.off_traj = o;    o += round256(p.rows0 * 4);
+  p.total = o;
+  return p;
+}
+
+size_t pg_rollout_run_workspace_bytes(const pg_config* cfg) {
+  if (validate_config(cfg) != PG_OK) return 0;
+  return make_run_plan(cfg).total;
+}
+
+int pg_rollout_run(pg_rollout* h, const pg_step_coef* step_coef, const pg_preview_coef* preview_coef,
+                   const float* x0, const void* const* vel_steps, const float* const* stage_scores,
+                   const float* final_rewards, void* workspace, size_t workspace_bytes,
+                   pg_rollout_outputs* out, void* stream) {
+  if (!h || !step_coef || !x0 || !vel_steps || !workspace || !out || !aligned16(workspace) ||
+      !aligned16(x0))
+    return PG_EINVAL;
+  const pg_config* cfg = &h->cfg;
+  const RunPlan pl = make_run_plan(cfg);
+  if (workspace_bytes < pl.total) return PG_EINVAL;
+  for (int s = 0; s < cfg->n_steps; ++s)
+    if (!vel_steps[s]) return PG_EINVAL;
+  for (int i = 0; i < cfg->n_stages; ++i)
+    if (!(stage_scores && stage_scores[i]) && !preview_coef) return PG_EINVAL;
+  unsigned char* ws = (unsigned char*)workspace;
+  float* d_x[2] = {(float*)(ws + pl.off_x[0]), (float*)(ws + pl.off_x[1])};
+  float* d_scores = (float*)(ws + pl.off_scores);
+  int32_t* d_keep = (int32_t*)(ws + pl.off_keep);
+  int32_t* d_src = (int32_t*)(ws + pl.off_src);
+  float* d_logp = (float*)(ws + pl.off_logp);
+  float* d_rewards = (float*)(ws + pl.off_rewards);
+  float* d_adv = (float*)(ws + pl.off_adv);
+  int32_t* d_traj = (int32_t*)(ws + pl.off_traj);
+
+  int rc = pg_rollout_reset(h, stream);
+  if (rc != PG_OK) return rc;
+  const float* x_cur = x0;       // read-only until the first step has written into the workspace
+  int cur = -1, stage = 0;       // cur: which workspace half holds x (-1: still x0)
+  size_t logp_off = 0, keep_off = 0;
+  for (int s = 0; s < cfg->n_steps; ++s) {
+    const int32_t* src = nullptr;
+    if (stage < cfg->n_stages && cfg->stage_step[stage] == s) {
+      const float* sc = (stage_scores && stage_scores[stage]) ? stage_scores[stage] : nullptr;
+      if (!sc) {
+        rc = pg_score(h, &preview_coef[stage], x_cur, vel_steps[s], d_scores, nullptr, stream);
+        if (rc != PG_OK) return rc;
+        sc = d_scores;
+      }
+      rc = pg_prune_ovf(h, stage, sc, d_keep + keep_off, d_src, nullptr, stream);
+      if (rc != PG_OK) return rc;
+      keep_off += (size_t)cfg->n_groups * h->k_cur;
+      src = d_src;
+      ++stage;
+    }
+    float* x_out;
+    if (cur < 0) { x_out = d_x[0]; }
+    else if (src) { x_out = d_x[cur ^ 1]; }
+    else { x_out = d_x[cur]; }
+    rc = pg_step(h, s, &step_coef[s], x_cur, vel_steps[s], src, x_out, d_logp + logp_off, stream);
+    if (rc != PG_OK) return rc;
+    if (cur < 0) cur = 0; else if (src) cur ^= 1;
+    x_cur = d_x[cur];
+    logp_off += (size_t)cfg->n_groups * h->k_cur;
+  }
+  const float* rw = final_rewards;
+  if (!rw) {
+    const pg_preview_coef id = {1.0, 0.0};
+    rc = pg_score(h, &id, x_cur, nullptr, d_rewards, nullptr, stream);
+    if (rc != PG_OK) return rc;
+    rw = d_rewards;
+  }
+  rc = pg_advantages(h, rw, d_adv, nullptr, nullptr, stream);
+  if (rc != PG_OK) return rc;
+  rc = pg_rollout_traj_ids(h, d_traj, stream);
+  if (rc != PG_OK) return rc;
+  out->x_final = d_x[cur];
+  out->logp = d_logp;
+  out->keep_idx = d_keep;
+  out->adv = d_adv;
+  out->rewards = rw;
+  out->traj_id = d_traj;
+  out->n_final = cfg->n_groups * h->k_cur;
+  out->n_logp = (int64_t)pl.total_logp;
+  out->n_keep = (int64_t)pl.total_keep;
+  return PG_OK;
+}
+
 }  // extern "C"

@@ -163,3 +163,63 @@ class Rollout:
         out.stage_var = list(self.sel_var)
         out.rewards, out.adv, out.mean, out.std = rw, self.adv, self.mean, self.std
         return out
+
+
+class NativeRollout:
+    """Whole rollouts through pg_rollout_run: one library call enqueues every launch of the
+    schedule on the current stream (device-resident inputs), optionally replayed as a CUDA graph
+    when the rollout is launch-bound."""
+
+    def __init__(self, ro: Rollout, step_coefs, preview_coefs, vel_steps, stage_scores=None):
+        self.ro = ro
+        self.args = B.RunArgs(step_coefs, preview_coefs, vel_steps, stage_scores)
+        self.ws = torch.empty(B.rollout_run_workspace_bytes(ro.cfg), dtype=torch.uint8, device=ro.dev)
+        self.graph = None
+        self.x0 = None
+
+    def _view(self, ptr: int, count: int, dtype: torch.dtype) -> torch.Tensor:
+        off = ptr - self.ws.data_ptr()
+        size = torch.empty(0, dtype=dtype).element_size()
+        return self.ws[off: off + count * size].view(dtype)
+
+    def run(self, x0: torch.Tensor, final_rewards: Optional[torch.Tensor] = None) -> RolloutOutput:
+        o = B.rollout_run(self.ro.h, self.args, x0, final_rewards, self.ws)
+        return self._outputs(o)
+
+    def capture(self, x0: torch.Tensor, final_rewards: Optional[torch.Tensor] = None) -> None:
+        """Records one rollout from x0 into a CUDA graph; replay() then re-runs it."""
+        self.x0 = x0
+        s = torch.cuda.Stream()
+        s.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(s):
+            B.rollout_run(self.ro.h, self.args, x0, final_rewards, self.ws)      # warm-up, loads kernels
+        torch.cuda.current_stream().wait_stream(s)
+        torch.cuda.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            self.out_struct = B.rollout_run(self.ro.h, self.args, x0, final_rewards, self.ws)
+
+    def replay(self) -> RolloutOutput:
+        self.graph.replay()
+        return self._outputs(self.out_struct)
+
+    def _outputs(self, o) -> RolloutOutput:
+        ro = self.ro
+        n, d = int(o.n_final), ro.d
+        logp_all = self._view(o.logp, int(o.n_logp), torch.float32)
+        keep_all = self._view(o.keep_idx, int(o.n_keep), torch.int32) if o.n_keep else None
+        out = RolloutOutput(x_final=self._view(o.x_final, n * d, torch.float32).view(n, d), logp=[],
+                            traj_id=self._view(o.traj_id, n, torch.int32))
+        off = 0
+        for rows in ro.rows_at:
+            out.logp.append(logp_all[off: off + rows])
+            off += rows
+        off = 0
+        for _, k in ro.stages:
+            out.stage_keep.append(keep_all[off: off + ro.G * k])
+            off += ro.G * k
+        out.adv = self._view(o.adv, n, torch.float32)
+        ws_lo, ws_hi = self.ws.data_ptr(), self.ws.data_ptr() + self.ws.numel()
+        if ws_lo <= o.rewards < ws_hi:
+            out.rewards = self._view(o.rewards, n, torch.float32)
+        return out

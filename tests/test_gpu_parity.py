@@ -597,3 +597,33 @@ def test_ovf_misaligned_and_ragged_score_rows(B):
             keep = torch.empty(G * k, dtype=torch.int32, device="cuda")
             B.ovf_select_batched(G, n, k, view, keep)
             np.testing.assert_array_equal(keep.cpu().numpy().reshape(G, k), ref_keep)
+
+
+def test_native_rollout_and_graph_replay_equal_the_stepwise_driver(B):
+    from paper_2512_15347_b200.rollout import NativeRollout
+    w = wl.scaled(wl.WORKLOADS["large"], n_groups=3, elems=8192 + 256)
+    inp = U.SharedInputs(w)
+    ro, out = U.run_gpu(w, inp)
+    want = (out.x_final.clone(), torch.cat(out.logp).clone(), torch.cat(out.stage_keep).clone(),
+            out.adv.clone(), out.traj_id.clone())
+    vels = [U.vel_to_dev(inp.vel_numpy(s, np.empty((w.n_groups * w.rows_before(s), 0))))
+            for s in range(w.n_steps)]
+    nat = NativeRollout(ro, [w.step_coef(s) for s in range(w.n_steps)],
+                        [w.preview_coef(s) for s, _ in w.stages], vels)
+    x0 = U.to_dev(inp.x0)
+
+    def check(o):
+        torch.cuda.synchronize()
+        assert torch.equal(o.x_final, want[0])
+        assert torch.equal(torch.cat(o.logp), want[1])
+        assert torch.equal(torch.cat(o.stage_keep), want[2])
+        assert torch.equal(o.adv, want[3])
+        assert torch.equal(o.traj_id, want[4])
+
+    check(nat.run(x0))
+    nat.capture(x0)
+    for _ in range(3):
+        nat.ws.zero_()                      # results must be rebuilt by the replay alone
+        check(nat.replay())
+    assert B.rollout_status(ro.h) == (w.n_groups * w.final_keep, w.n_steps, 0)
+    ro.close()
