@@ -173,7 +173,7 @@ int pg_prune_ovf(pg_rollout *h, int32_t stage, const float *scores, int32_t *kee
                  int32_t *src_rows, float *sel_var, void *stream);
 
 /*
- * Uniform-subsampling baseline (Section 4.1, Fig. 1b: "uniformly subsampling k < G candidates"):
+ * Uniform-subsampling baseline (Section 4.1, Fig. 1b: k of the G candidates drawn uniformly at random):
  * same contract and cursor effects as pg_prune_ovf, but the k survivors of each group are a
  * uniformly random subset, independent of any score.  Reproducible: slot i of group g draws the
  * first Philox4x32-10 word of counter (i, stage, group_offset + g, stream id 4) under the
@@ -193,8 +193,8 @@ int pg_group_stats(int32_t n_groups, int32_t n, const float *scores, float delta
 
 /*
  * Survivor compaction of a caller-side row array after the most recent
- * pg_prune_ovf (Section 5.1: pruned trajectories "incur no further SDE
- * steps"): dst row g*k + p = src row g*K_prev + keep_idx[g*k + p]; order and
+ * pg_prune_ovf (Section 5.1: a pruned trajectory is never stepped again, so
+ * only survivors are carried on): dst row g*k + p = src row g*K_prev + keep_idx[g*k + p]; order and
  * count are preserved.  row_bytes > 0; rows need only be byte-aligned, 16-byte
  * aligned rows are moved with 128-bit accesses.  dst must not overlap src.
  */
@@ -212,7 +212,8 @@ int pg_advantages(pg_rollout *h, const float *rewards, float *adv, float *mean, 
 
 /*
  * Policy update on the survivors, forward part for one step (Eq. "ratio_method": pi_theta is
- * the Gaussian policy induced by Eq. "euler_method"; KL term of Eq. "pro_grpo_method").
+ * the Gaussian transition density of the update of Eq. "euler_method"; KL term of Eq.
+ * "pro_grpo_method").
  * For each of the n_active rows, with m = c_x x + c_v vel and s = noise_std > 0:
  *     logp_out[i] = -1/2 sum_e ((x_next_e - m_e)/s)^2 - d/2 ln(2 pi s^2)        (/ d if logp_mean)
  *     kl_out[i]   = KL(N(m, s^2 I) || N(m_ref, s^2 I)) = c_v^2 sum_e (vel_e - vel_ref_e)^2 / (2 s^2)

@@ -330,8 +330,8 @@ static double arithmetic_value(float s)
 /*
  * OVF for any group size (Eq. "ovf", and its in-process form in Section 5.1).
  * The variance of a set is a convex quadratic in each member, so a maximiser
- * always has the shape "the j lowest and the k-j highest scores" ("selecting
- * from the reward extremes", Fig. 1c).  Steps:
+ * always has the shape "the j lowest and the k-j highest scores" (the subset
+ * sits at both ends of the score range, as Fig. 1c illustrates).  Steps:
  *   1. order the slots by (score, slot);
  *   2. centre on the score at order position n/2 (keeps the sums small);
  *   3. running sums of c and c*c from the low end (L1, L2) and from the high
@@ -418,8 +418,8 @@ int og_ovf_select_groups(int n_groups, int n, int k, const float *scores,
 /* ------------------------------------------------------------------ */
 
 /*
- * Early termination (Section 5.1: pruned trajectories "incur no further SDE
- * steps"): the survivors of each group become a dense block, in ascending
+ * Early termination (Section 5.1: a pruned trajectory is never stepped
+ * again): the survivors of each group become a dense block, in ascending
  * slot order.  Row g*k + p of dst is row g*n_prev + keep_idx[g*k + p] of src.
  */
 int og_compact_rows(int n_groups, int n_prev, int k, const int32_t *keep_idx,

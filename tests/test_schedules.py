@@ -1,6 +1,6 @@
 """Coefficient builders against the mathematics they encode: for Gaussian data the exact network
 prediction is linear, so a correct sampler must reproduce the data distribution (the SDE
-conversions "maintain consistent marginal distributions", Section 3.2)."""
+conversions of Section 3.2 are meant to leave the marginal distributions unchanged)."""
 import math
 
 import numpy as np
