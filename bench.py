@@ -416,29 +416,38 @@ def run_e2e(B, wl, w, wr, rank, dist, dev, args):
     cfg = B.make_config(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed,
                         B.VEL_BF16 if w.vel_dtype == "bf16" else B.VEL_F32, adv_eps=w.adv_eps,
                         group_offset=rank * w.n_groups)  # = sharding.weak_shard(...)[0]
-    ws = torch.empty(B.rollout_host_workspace_bytes(cfg), dtype=torch.uint8, device=dev)
-    dt = torch.bfloat16 if w.vel_dtype == "bf16" else torch.float32
-    # host inputs: pinned; filled from a seeded CPU generator block by block (content does not
-    # affect timing, but the bytes are real N(0,1) draws)
-    g = torch.Generator().manual_seed(1234 + rank)
-    x0 = torch.empty(w.n_groups * w.n_expand, w.elems, dtype=torch.float32).pin_memory()
-    block = torch.randn(64, w.elems, generator=g)
-    for i in range(0, x0.shape[0], 64):
-        x0[i:i + 64] = block[: x0.shape[0] - i].roll(i // 64, 1)
-    vels = []
-    vblock = torch.randn(64, w.elems, generator=g).to(dt)
-    for s in range(w.n_steps):
-        rows = w.n_groups * w.rows_before(s)
-        v = torch.empty(rows, w.elems, dtype=dt).pin_memory()
-        for i in range(0, rows, 64):
-            v[i:i + 64] = vblock[: rows - i].roll(s * 64 + i // 64, 1)
-        vels.append(v)
-    K = w.final_keep
-    x_final = torch.empty(w.n_groups * K, w.elems).pin_memory()
-    logp = torch.empty(w.traj_steps).pin_memory()
-    keep = torch.empty(sum(w.n_groups * k for _, k in w.stages), dtype=torch.int32).pin_memory()
-    adv = torch.empty(w.n_groups * K).pin_memory()
-    ids = torch.empty(w.n_groups * K, dtype=torch.int32).pin_memory()
+    from paper_2512_15347_b200 import sharding
+    # every rank pins its own copy of the inputs (26 GB for the large workload): if any rank cannot
+    # get them, all ranks skip the end-to-end leg together
+    ok, why = 1.0, ""
+    try:
+        ws = torch.empty(B.rollout_host_workspace_bytes(cfg), dtype=torch.uint8, device=dev)
+        dt = torch.bfloat16 if w.vel_dtype == "bf16" else torch.float32
+        # host inputs: pinned; filled from a seeded CPU generator block by block (content does not
+        # affect timing, but the bytes are real N(0,1) draws)
+        g = torch.Generator().manual_seed(1234 + rank)
+        x0 = torch.empty(w.n_groups * w.n_expand, w.elems, dtype=torch.float32).pin_memory()
+        block = torch.randn(64, w.elems, generator=g)
+        for i in range(0, x0.shape[0], 64):
+            x0[i:i + 64] = block[: x0.shape[0] - i].roll(i // 64, 1)
+        vels = []
+        vblock = torch.randn(64, w.elems, generator=g).to(dt)
+        for s in range(w.n_steps):
+            rows = w.n_groups * w.rows_before(s)
+            v = torch.empty(rows, w.elems, dtype=dt).pin_memory()
+            for i in range(0, rows, 64):
+                v[i:i + 64] = vblock[: rows - i].roll(s * 64 + i // 64, 1)
+            vels.append(v)
+        K = w.final_keep
+        x_final = torch.empty(w.n_groups * K, w.elems).pin_memory()
+        logp = torch.empty(w.traj_steps).pin_memory()
+        keep = torch.empty(sum(w.n_groups * k for _, k in w.stages), dtype=torch.int32).pin_memory()
+        adv = torch.empty(w.n_groups * K).pin_memory()
+        ids = torch.empty(w.n_groups * K, dtype=torch.int32).pin_memory()
+    except Exception as e:            # out of host or device memory
+        ok, why = 0.0, f"{type(e).__name__}: {e}"[:200]
+    if -sharding.max_over_ranks(-ok, dist, dev) < 1.0:
+        return {"value": None, "unit": UNIT, "unavailable": why or "another rank could not allocate its buffers"}
     coefs = [w.step_coef(s) for s in range(w.n_steps)]
     pcoefs = [w.preview_coef(s) for s, _ in w.stages]
 
@@ -456,7 +465,6 @@ def run_e2e(B, wl, w, wr, rank, dist, dev, args):
         call()
     b.record()
     torch.cuda.synchronize()
-    from paper_2512_15347_b200 import sharding
     ms = sharding.max_over_ranks(a.elapsed_time(b), dist, dev)
     world = 1 if dist is None else dist.get_world_size()
     h2d = x0.numel() * 4 + sum(v.numel() * v.element_size() for v in vels)
