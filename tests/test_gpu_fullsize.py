@@ -11,7 +11,7 @@ from tests import util as U
 
 pytestmark = pytest.mark.gpu
 
-SAMPLED_GROUPS = (0, 37, 63)
+SAMPLED_GROUPS = (0, 5, 17, 31, 37, 50, 62, 63)
 
 
 def test_large_workload_sampled_groups_match_oracle():
@@ -107,3 +107,20 @@ def test_ovf_microbench_shape_matches_oracle():
     ref_adv, _, _ = oracle.advantages(ref_kept, 1e-6)
     np.testing.assert_allclose(adv.cpu().numpy().reshape(G, k), ref_adv, rtol=1e-5, atol=1e-6)
     assert int(st.item()) == 0
+
+
+def test_sd3_workload_full_size_matches_oracle_everywhere():
+    """The SD3 / FLUX-shaped workload (16 groups x 48 -> 24 -> 12, 28 steps, 16x128x128 latents,
+    external clustered scores) is small enough for the oracle to follow every trajectory."""
+    from paper_2512_15347_b200 import binding as B
+    w = wl.WORKLOADS["sd3"]
+    inp = U.SharedInputs(w)
+    ref = U.run_oracle(w, inp)
+    ro, out = U.run_gpu(w, inp)
+    lp_err, x_err = U.compare_rollouts(w, ref, out)
+    assert B.rollout_status(ro.h) == (w.n_groups * w.final_keep, w.n_steps, 0)
+    # selection statistics the method is about: the kept subset is more spread out than the group
+    for i, (s, k) in enumerate(w.stages):
+        sc = ref.stage_scores[i].astype(np.float64)
+        assert np.all(ref.stage_var[i] >= sc.var(axis=1) - 1e-12)
+    ro.close()
