@@ -1,13 +1,11 @@
-// Optimal Variance Filtering (Eq. "ovf"), survivor index compaction and group-relative
-// advantages (Eq. "advK").
+// Optimal Variance Filtering (Eq. "ovf"), survivor index compaction, group-relative advantages
+// (Eq. "advK"), clustering diagnostics and the uniform-subsampling baseline.
 //
-// One CTA per group.  The scores of the group are staged in shared memory as 64-bit keys
-// (order-preserving image of the fp32 score in the high word, slot in the low word), so
-// every key is distinct and the total order (score, slot) is a plain integer order.  Each
-// element finds its rank by counting smaller keys; the sorted values then give the running
-// sums from both ends, the k+1 candidate variances "j lowest + (k-j) highest" are evaluated
-// in fp64 with explicitly rounded operations, and the kept slots are written in ascending
-// slot order through a ballot/popcount prefix sum.
+// Selection: one warp per group; the scores become order-preserving 32-bit keys, are sorted in
+// registers, every element finds its rank in the total order (score, slot), the running sums
+// from both ends give the k+1 candidate variances "j lowest + (k-j) highest" in fp64 with
+// explicitly rounded operations, and the kept slots are written in ascending slot order through
+// a popcount prefix sum.
 #include "pg_common.cuh"
 #include <float.h>
 
@@ -46,209 +44,10 @@ __device__ __forceinline__ double arithmetic_value(float s) {
   return (double)s;
 }
 
-__global__ void __launch_bounds__(kOvfThreads)
-ovf_select_kernel(const __grid_constant__ OvfParams p) {
-  extern __shared__ __align__(16) unsigned char smem[];
-  const int n = p.n, k = p.k;
-  unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem);       // [n]
-  double* L1 = reinterpret_cast<double*>(keys + n);                             // [k+1] each
-  double* L2 = L1 + (k + 1);
-  double* H1 = L2 + (k + 1);
-  double* H2 = H1 + (k + 1);
-  float* sorted = reinterpret_cast<float*>(H2 + (k + 1));                       // [n]
-  __shared__ double red_m[kOvfThreads / 32];
-  __shared__ int red_j[kOvfThreads / 32];
-  __shared__ int warp_cnt[kOvfThreads / 32];
-  __shared__ int best_j_s;
-  __shared__ double stat_s[2];
-
-  const int g = blockIdx.x;
-  const int tid = threadIdx.x;
-  const float* sc = p.scores + (size_t)g * n;
-
-  // 1. stage keys
-  bool bad = false;
-  for (int i = tid; i < n; i += kOvfThreads) {
-    const float s = sc[i];
-    bad |= !(fabsf(s) <= FLT_MAX);
-    keys[i] = ((unsigned long long)order_key(s) << 32) | (unsigned int)i;
-    sorted[i] = 0.f;
-  }
-  if (bad && p.status) atomicOr(p.status, 1);
-  __syncthreads();
-
-  // 2. rank by counting; ranks are a permutation because keys are distinct
-  constexpr int kMaxPerThread = PG_MAX_GROUP / kOvfThreads;
-  int rank[kMaxPerThread];
-#pragma unroll
-  for (int t = 0; t < kMaxPerThread; ++t) {
-    const int i = tid + t * kOvfThreads;
-    rank[t] = 0;
-    if (i < n) {
-      const unsigned long long mine = keys[i];
-      int r = 0;
-      for (int j = 0; j < n; ++j) r += (keys[j] < mine) ? 1 : 0;
-      rank[t] = r;
-      sorted[r] = sc[i];
-    }
-  }
-  __syncthreads();
-
-  // 3. running sums from both ends, serial and in order (fp64, no contraction)
-  if (tid == 0 || tid == 32) {
-    const double pivot = arithmetic_value(sorted[n / 2]);
-    double a1 = 0.0, a2 = 0.0;
-    if (tid == 0) {
-      L1[0] = 0.0; L2[0] = 0.0;
-      for (int j = 1; j <= k; ++j) {
-        const double c = __dsub_rn(arithmetic_value(sorted[j - 1]), pivot);
-        a1 = __dadd_rn(a1, c);
-        a2 = __dadd_rn(a2, __dmul_rn(c, c));
-        L1[j] = a1; L2[j] = a2;
-      }
-    } else {
-      H1[0] = 0.0; H2[0] = 0.0;
-      for (int m = 1; m <= k; ++m) {
-        const double c = __dsub_rn(arithmetic_value(sorted[n - m]), pivot);
-        a1 = __dadd_rn(a1, c);
-        a2 = __dadd_rn(a2, __dmul_rn(c, c));
-        H1[m] = a1; H2[m] = a2;
-      }
-    }
-  }
-  __syncthreads();
-
-  // 4. candidates j = 0..k; keep the largest j among the maxima
-  double best_m = -1.0;
-  int best_j = -1;
-  for (int j = tid; j <= k; j += kOvfThreads) {
-    const double S = __dadd_rn(L1[j], H1[k - j]);
-    const double Q = __dadd_rn(L2[j], H2[k - j]);
-    const double M = __dsub_rn(__dmul_rn((double)k, Q), __dmul_rn(S, S));
-    if (best_j < 0 || M >= best_m) { best_m = M; best_j = j; }
-  }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const double om = __shfl_xor_sync(0xFFFFFFFFu, best_m, o);
-    const int oj = __shfl_xor_sync(0xFFFFFFFFu, best_j, o);
-    if (oj >= 0 && (best_j < 0 || om > best_m || (om == best_m && oj > best_j))) {
-      best_m = om; best_j = oj;
-    }
-  }
-  if ((tid & 31) == 0) { red_m[tid >> 5] = best_m; red_j[tid >> 5] = best_j; }
-  __syncthreads();
-  if (tid == 0) {
-    double bm = red_m[0];
-    int bj = red_j[0];
-    for (int w = 1; w < kOvfThreads / 32; ++w) {
-      const double om = red_m[w];
-      const int oj = red_j[w];
-      if (oj >= 0 && (bj < 0 || om > bm || (om == bm && oj > bj))) { bm = om; bj = oj; }
-    }
-    best_j_s = bj;
-    if (p.sel_var) p.sel_var[g] = (float)(bm / ((double)k * (double)k));
-  }
-  __syncthreads();
-  const int jstar = best_j_s;
-  const int high_from = n - (k - jstar);     // ranks >= high_from are kept from the top
-
-  // 5. kept slots in ascending slot order
-  int running = 0;
-  double sum_kept = 0.0;
-#pragma unroll
-  for (int t = 0; t < kMaxPerThread; ++t) {
-    const int base = t * kOvfThreads;
-    if (base >= n) break;
-    const int i = base + tid;
-    const bool keep = (i < n) && (rank[t] < jstar || rank[t] >= high_from);
-    const unsigned int bal = __ballot_sync(0xFFFFFFFFu, keep);
-    if ((tid & 31) == 0) warp_cnt[tid >> 5] = __popc(bal);
-    __syncthreads();
-    int before = 0, total = 0;
-#pragma unroll
-    for (int w = 0; w < kOvfThreads / 32; ++w) {
-      const int c = warp_cnt[w];
-      if (w < (tid >> 5)) before += c;
-      total += c;
-    }
-    if (keep) {
-      const int pos = running + before + __popc(bal & ((1u << (tid & 31)) - 1u));
-      const size_t o = (size_t)g * k + pos;
-      p.keep_idx[o] = i;
-      if (p.src_rows) p.src_rows[o] = g * n + i;
-      if (p.traj_out) p.traj_out[o] = p.traj_in[(size_t)g * n + i];
-      const float s = sc[i];
-      if (p.kept_scores) p.kept_scores[o] = s;
-      sum_kept += (double)s;
-    }
-    running += total;
-    __syncthreads();
-  }
-
-  // 6. optional advantages of the kept scores (Eq. "advK" on the selected set)
-  if (p.adv) {
-    double v = warp_sum(sum_kept);
-    if ((tid & 31) == 0) red_m[tid >> 5] = v;
-    __syncthreads();
-    if (tid == 0) {
-      double s = 0.0;
-      for (int w = 0; w < kOvfThreads / 32; ++w) s += red_m[w];
-      stat_s[0] = s / (double)k;
-    }
-    __syncthreads();
-    const double mu = stat_s[0];
-    double sq = 0.0;
-#pragma unroll
-    for (int t = 0; t < kMaxPerThread; ++t) {
-      const int i = t * kOvfThreads + tid;
-      if (i < n && (rank[t] < jstar || rank[t] >= high_from)) {
-        const double dlt = (double)sc[i] - mu;
-        sq += dlt * dlt;
-      }
-    }
-    v = warp_sum(sq);
-    __syncthreads();
-    if ((tid & 31) == 0) red_m[tid >> 5] = v;
-    __syncthreads();
-    if (tid == 0) {
-      double s = 0.0;
-      for (int w = 0; w < kOvfThreads / 32; ++w) s += red_m[w];
-      stat_s[1] = sqrt(s / (double)k);
-    }
-    __syncthreads();
-    const double denom = stat_s[1] + (double)p.adv_eps;
-    // kept entries were written above by the same threads; recompute their positions
-    running = 0;
-#pragma unroll
-    for (int t = 0; t < kMaxPerThread; ++t) {
-      const int base = t * kOvfThreads;
-      if (base >= n) break;
-      const int i = base + tid;
-      const bool keep = (i < n) && (rank[t] < jstar || rank[t] >= high_from);
-      const unsigned int bal = __ballot_sync(0xFFFFFFFFu, keep);
-      if ((tid & 31) == 0) warp_cnt[tid >> 5] = __popc(bal);
-      __syncthreads();
-      int before = 0, total = 0;
-#pragma unroll
-      for (int w = 0; w < kOvfThreads / 32; ++w) {
-        const int c = warp_cnt[w];
-        if (w < (tid >> 5)) before += c;
-        total += c;
-      }
-      if (keep) {
-        const int pos = running + before + __popc(bal & ((1u << (tid & 31)) - 1u));
-        p.adv[(size_t)g * k + pos] = (float)(((double)sc[i] - mu) / denom);
-      }
-      running += total;
-      __syncthreads();
-    }
-  }
-}
-
-// ---------------------------------------------------------------- groups of up to 256 scores
+// ---------------------------------------------------------------- selection kernel
 //
-// One warp per group, E = 1, 2, 4 or 8 scores per lane (n <= 32 * E); the four warps of a CTA
-// only meet once, for the staging of their score rows.
+// One warp per group, E = 1, 2, 4, 8, 16 or 32 scores per lane (n <= 32 * E <= 1024); the warps
+// of a CTA (four, or one for the widest groups) only meet once, for the staging of their rows.
 //  0. The CTA's score rows are staged in shared memory by one bulk asynchronous copy
 //     (cp.async.bulk, completion on an mbarrier, bounded wait) when source and size are
 //     16-byte aligned, else read with ordinary loads.
@@ -263,7 +62,8 @@ ovf_select_kernel(const __grid_constant__ OvfParams p) {
 //     rounded operations - the same operations in the same order as a plain serial loop.
 //  4. k+1 candidates, argmax with the "largest j" tie rule, membership by rank; every lane holds
 //     its scores in slot order, so a popcount prefix over lanes gives ascending slot order.
-constexpr int kOvfWarpsPerCta = 4;
+// warps (= groups) per CTA: four while the per-warp shared memory allows it, one for wide groups
+template <int E> struct OvfWarps { static constexpr int value = (E <= 8) ? 4 : 1; };
 constexpr int kBulkWaitLimit = 1 << 14;   // mbarrier try_wait attempts before giving up
 
 __device__ __forceinline__ float key_to_score(uint32_t key) {
@@ -272,9 +72,10 @@ __device__ __forceinline__ float key_to_score(uint32_t key) {
 }
 
 template <int E>
-__global__ void __launch_bounds__(kOvfWarpsPerCta * 32)
+__global__ void __launch_bounds__(OvfWarps<E>::value * 32)
 ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
   constexpr int N = 32 * E;
+  constexpr int kOvfWarpsPerCta = OvfWarps<E>::value;
   extern __shared__ __align__(16) unsigned char smem[];
   __shared__ __align__(8) unsigned long long stage_bar;
   const int n = p.n, k = p.k;
@@ -518,6 +319,7 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
 template <int E>
 static void launch_ovf_warp(const OvfParams& p, int n_groups, cudaStream_t stream) {
   const size_t per_warp = (size_t)(p.k + 1) * 4 * sizeof(double) + (size_t)(32 * E) * 2 * sizeof(uint32_t);
+  constexpr int kOvfWarpsPerCta = OvfWarps<E>::value;
   const size_t stage = (size_t)kOvfWarpsPerCta * 32 * E * sizeof(float);
   const int ctas = (n_groups + kOvfWarpsPerCta - 1) / kOvfWarpsPerCta;
   ovf_warp_kernel<E><<<ctas, kOvfWarpsPerCta * 32, stage + per_warp * kOvfWarpsPerCta, stream>>>(p, n_groups);
@@ -545,10 +347,8 @@ int launch_ovf(int n_groups, int n, int k, const float* scores, int32_t* keep_id
   else if (n <= 64)  launch_ovf_warp<2>(p, n_groups, stream);
   else if (n <= 128) launch_ovf_warp<4>(p, n_groups, stream);
   else if (n <= 256) launch_ovf_warp<8>(p, n_groups, stream);
-  else {
-    const size_t smem = (size_t)n * 8 + (size_t)(k + 1) * 4 * 8 + (size_t)n * 4;
-    ovf_select_kernel<<<n_groups, kOvfThreads, smem, stream>>>(p);
-  }
+  else if (n <= 512) launch_ovf_warp<16>(p, n_groups, stream);
+  else launch_ovf_warp<32>(p, n_groups, stream);
   PG_LAUNCH_CHECK();
   return PG_OK;
 }
