@@ -54,6 +54,7 @@ extern "C" {
 #define PG_ENONFINITE (-4)  /* reported by pg_rollout_status(): non-finite scores seen */
 #define PG_ETIMEOUT   (-5)  /* reported by pg_rollout_status(): a bounded device wait expired */
 #define PG_ENOMEM     (-6)  /* host or device allocation for the handle failed         */
+#define PG_EINDEX     (-8)  /* reported by pg_rollout_status(): a gather index was out of range */
 #define PG_ECAPACITY  (-7)  /* request larger than a fixed built-in buffer (pg_score_static) */
 
 #define PG_VEL_F32  0
@@ -108,9 +109,12 @@ int pg_rollout_reset(pg_rollout *h, void *stream);
 /*
  * Synchronises the device and reports the host-side cursor (trajectories
  * active in total, next step index) and the device status word (bit 0:
- * non-finite score seen by pg_prune_ovf, bit 1: a bounded wait expired).
- * Any out pointer may be NULL.  Returns PG_ENONFINITE / PG_ETIMEOUT if the
- * corresponding bit is set, else PG_OK.
+ * non-finite score seen by pg_prune_ovf, bit 1: a bounded wait expired, bit 2:
+ * a src_rows / keep_idx entry given to pg_step / pg_compact was out of range -
+ * such an entry is never dereferenced: pg_step computes that row from row 0,
+ * pg_compact leaves it unwritten).  Any out pointer may be NULL.  Returns
+ * PG_EINDEX / PG_ETIMEOUT / PG_ENONFINITE if the corresponding bit is set (in
+ * that order of precedence), else PG_OK.
  */
 int pg_rollout_status(pg_rollout *h, int32_t *n_active, int32_t *next_step, int32_t *device_status);
 

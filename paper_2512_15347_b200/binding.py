@@ -14,7 +14,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libprogrpo.so")
 
-OK, EINVAL, ESTATE, ECUDA, ENONFINITE, ETIMEOUT, ENOMEM, ECAPACITY = 0, -1, -2, -3, -4, -5, -6, -7
+OK, EINVAL, ESTATE, ECUDA, ENONFINITE, ETIMEOUT, ENOMEM, ECAPACITY, EINDEX = 0, -1, -2, -3, -4, -5, -6, -7, -8
 STATIC_MAX_ROWS, STATIC_MAX_PARTIALS = 8192, 65536
 VEL_F32, VEL_BF16 = 0, 1
 MAX_GROUP = 1024
@@ -167,7 +167,7 @@ def rollout_status(h: int, raise_on_flags: bool = True):
     """(n_active, next_step, device_status); synchronises the device."""
     a, b, c = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
     rc = lib().pg_rollout_status(h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
-    if rc != OK and (raise_on_flags or rc not in (ENONFINITE, ETIMEOUT)):
+    if rc != OK and (raise_on_flags or rc not in (ENONFINITE, ETIMEOUT, EINDEX)):
         raise PgError(rc, "pg_rollout_status")
     return a.value, b.value, c.value
 

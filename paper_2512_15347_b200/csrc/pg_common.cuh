@@ -242,7 +242,8 @@ struct RowScratch {
 int launch_step(int n_rows, int elems, int vel_dtype, const float* x_in, const void* vel,
                 const int32_t* src_rows, const int32_t* traj_id, float* x_out, float* logp_out,
                 uint64_t seed, int32_t step, double c_x, double c_v, double noise_std,
-                int logp_mean, RowScratch scratch, cudaStream_t stream);
+                int logp_mean, RowScratch scratch, cudaStream_t stream, int rows_in = 0,
+                int32_t* status = nullptr);
 
 int launch_score(int n_rows, int elems, int vel_dtype, const float* x, const void* vel,
                  double p_x, double p_v, float* scores_out, float* preview_out,
@@ -280,7 +281,7 @@ int launch_advantages(int n_groups, int K, const float* rewards, float eps, floa
                       float* mean, float* std_out, cudaStream_t stream);
 
 int launch_compact(int n_groups, int n_prev, int k, const int32_t* keep_idx, const void* src,
-                   void* dst, size_t row_bytes, cudaStream_t stream);
+                   void* dst, size_t row_bytes, cudaStream_t stream, int32_t* status = nullptr);
 
 int launch_iota(int32_t* dst, int n, int32_t base, cudaStream_t stream);
 

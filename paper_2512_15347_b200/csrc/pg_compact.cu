@@ -11,11 +11,15 @@ constexpr size_t kCompactPiece = 32768;   // bytes per CTA
 template <typename T>
 __global__ void __launch_bounds__(kCompactThreads)
 compact_kernel(const int32_t* keep_idx, const unsigned char* src, unsigned char* dst,
-               size_t row_bytes, int n_prev, int k, int pieces) {
+               size_t row_bytes, int n_prev, int k, int pieces, int32_t* status) {
   const int row = blockIdx.x / pieces;
   const int piece = blockIdx.x - row * pieces;
   const int g = row / k;
   const int slot = keep_idx[row];
+  if ((unsigned int)slot >= (unsigned int)n_prev) {       // never dereference a bad slot
+    if (threadIdx.x == 0 && piece == 0 && status) atomicOr(status, 4);
+    return;
+  }
   const size_t begin = (size_t)piece * kCompactPiece;
   const size_t end = (begin + kCompactPiece < row_bytes) ? begin + kCompactPiece : row_bytes;
   const T* s = reinterpret_cast<const T*>(src + ((size_t)g * n_prev + slot) * row_bytes + begin);
@@ -27,16 +31,20 @@ compact_kernel(const int32_t* keep_idx, const unsigned char* src, unsigned char*
 // Narrow rows (a few bytes, e.g. one fp32 per trajectory): one thread per row.
 template <typename T>
 __global__ void compact_small_kernel(const int32_t* keep_idx, const T* src, T* dst, int n_rows,
-                                     int n_prev, int k, int per_row) {
+                                     int n_prev, int k, int per_row, int32_t* status) {
   const int row = blockIdx.x * blockDim.x + threadIdx.x;
   if (row >= n_rows) return;
   const int g = row / k;
+  if ((unsigned int)keep_idx[row] >= (unsigned int)n_prev) {
+    if (status) atomicOr(status, 4);
+    return;
+  }
   const size_t s = ((size_t)g * n_prev + keep_idx[row]) * per_row;
   for (int i = 0; i < per_row; ++i) dst[(size_t)row * per_row + i] = src[s + i];
 }
 
 int launch_compact(int n_groups, int n_prev, int k, const int32_t* keep_idx, const void* src,
-                   void* dst, size_t row_bytes, cudaStream_t stream) {
+                   void* dst, size_t row_bytes, cudaStream_t stream, int32_t* status) {
   const long long rows = (long long)n_groups * k;
   if (rows == 0) return PG_OK;
   const uintptr_t a = (uintptr_t)src | (uintptr_t)dst | (uintptr_t)row_bytes;
@@ -44,10 +52,10 @@ int launch_compact(int n_groups, int n_prev, int k, const int32_t* keep_idx, con
     const unsigned blocks = (unsigned)((rows + 255) / 256);
     if ((a & 3) == 0)
       compact_small_kernel<uint32_t><<<blocks, 256, 0, stream>>>(
-          keep_idx, (const uint32_t*)src, (uint32_t*)dst, (int)rows, n_prev, k, (int)(row_bytes / 4));
+          keep_idx, (const uint32_t*)src, (uint32_t*)dst, (int)rows, n_prev, k, (int)(row_bytes / 4), status);
     else
       compact_small_kernel<unsigned char><<<blocks, 256, 0, stream>>>(
-          keep_idx, (const unsigned char*)src, (unsigned char*)dst, (int)rows, n_prev, k, (int)row_bytes);
+          keep_idx, (const unsigned char*)src, (unsigned char*)dst, (int)rows, n_prev, k, (int)row_bytes, status);
     PG_LAUNCH_CHECK();
     return PG_OK;
   }
@@ -57,11 +65,11 @@ int launch_compact(int n_groups, int n_prev, int k, const int32_t* keep_idx, con
   const unsigned char* s = (const unsigned char*)src;
   unsigned char* d = (unsigned char*)dst;
   if ((a & 15) == 0)
-    compact_kernel<uint4><<<(unsigned)blocks, kCompactThreads, 0, stream>>>(keep_idx, s, d, row_bytes, n_prev, k, pieces);
+    compact_kernel<uint4><<<(unsigned)blocks, kCompactThreads, 0, stream>>>(keep_idx, s, d, row_bytes, n_prev, k, pieces, status);
   else if ((a & 3) == 0)
-    compact_kernel<uint32_t><<<(unsigned)blocks, kCompactThreads, 0, stream>>>(keep_idx, s, d, row_bytes, n_prev, k, pieces);
+    compact_kernel<uint32_t><<<(unsigned)blocks, kCompactThreads, 0, stream>>>(keep_idx, s, d, row_bytes, n_prev, k, pieces, status);
   else
-    compact_kernel<unsigned char><<<(unsigned)blocks, kCompactThreads, 0, stream>>>(keep_idx, s, d, row_bytes, n_prev, k, pieces);
+    compact_kernel<unsigned char><<<(unsigned)blocks, kCompactThreads, 0, stream>>>(keep_idx, s, d, row_bytes, n_prev, k, pieces, status);
   PG_LAUNCH_CHECK();
   return PG_OK;
 }

@@ -141,6 +141,7 @@ int pg_rollout_status(pg_rollout* h, int32_t* n_active, int32_t* next_step, int3
   if (n_active) *n_active = h->cfg.n_groups * h->k_cur;
   if (next_step) *next_step = h->next_step;
   if (device_status) *device_status = st;
+  if (st & 4) return PG_EINDEX;
   if (st & 2) return PG_ETIMEOUT;
   if (st & 1) return PG_ENONFINITE;
   return PG_OK;
@@ -161,7 +162,8 @@ int pg_step(pg_rollout* h, int32_t step, const pg_step_coef* coef, const float* 
   const int rc = pg::launch_step(rows, h->cfg.elems, h->cfg.vel_dtype, x_in, vel, src_rows,
                                  h->d_traj[h->traj_cur], x_out, logp_out, h->cfg.seed, step,
                                  coef->c_x, coef->c_v, coef->noise_std, h->cfg.logp_mean, scratch,
-                                 (cudaStream_t)stream);
+                                 (cudaStream_t)stream,
+                                 src_rows ? h->cfg.n_groups * h->k_prev : rows, h->d_status);
   if (rc == PG_OK) h->next_step = step + 1;
   return rc;
 }
@@ -240,7 +242,7 @@ int pg_compact(pg_rollout* h, const int32_t* keep_idx, const void* src, void* ds
   const uintptr_t s = (uintptr_t)src, d = (uintptr_t)dst;
   if (s < d + dst_bytes && d < s + src_bytes) return PG_EINVAL;   // overlap
   return pg::launch_compact(h->cfg.n_groups, h->k_prev, h->k_cur, keep_idx, src, dst, row_bytes,
-                            (cudaStream_t)stream);
+                            (cudaStream_t)stream, h->d_status);
 }
 
 int pg_advantages(pg_rollout* h, const float* rewards, float* adv, float* mean, float* std,
@@ -328,6 +330,7 @@ const char* pg_strerror(int code) {
     case PG_ENONFINITE: return "non-finite scores were seen by the selection";
     case PG_ETIMEOUT: return "a bounded device-side wait expired";
     case PG_ENOMEM: return "out of memory";
+    case PG_EINDEX: return "a gather index (src_rows / keep_idx) was out of range; the rows were not read";
     case PG_ECAPACITY: return "request exceeds the capacity of a fixed built-in buffer";
     default: return "unknown error code";
   }
@@ -497,7 +500,7 @@ int pg_rollout_host(const pg_config* cfg, const pg_step_coef* step_coef,
   PG_TRY_CUDA(cudaStreamSynchronize(compute));
   int32_t st = 0;
   PG_TRY_CUDA(cudaMemcpy(&st, h->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost));
-  return cleanup((st & 2) ? PG_ETIMEOUT : (st & 1) ? PG_ENONFINITE : PG_OK);
+  return cleanup((st & 4) ? PG_EINDEX : (st & 2) ? PG_ETIMEOUT : (st & 1) ? PG_ENONFINITE : PG_OK);
 #undef PG_TRY
 #undef PG_TRY_CUDA
 }

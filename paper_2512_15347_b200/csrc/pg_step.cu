@@ -21,6 +21,8 @@ struct StepParams {
   float* logp_out;
   float* partials;
   unsigned int* tickets;
+  int32_t* status;        // device status word (bit 2: gather index out of range) or null
+  int rows_in;            // rows of x_in / vel that src_rows may address
   int quads_per_row;      // d / 4
   int chunk_quads;        // quads per CTA
   int chunks;             // CTAs per row
@@ -102,7 +104,13 @@ step_kernel(const __grid_constant__ StepParams p) {
   using VReg = typename VelReg<VelT>::type;
   const int row = blockIdx.x / p.chunks;
   const int chunk = blockIdx.x - row * p.chunks;
-  const int src = p.src_rows ? p.src_rows[row] : row;
+  int src = p.src_rows ? p.src_rows[row] : row;
+  if ((unsigned int)src >= (unsigned int)p.rows_in) {
+    // a gather index outside the input: never dereferenced; the row is computed from row 0 so
+    // that the reduction protocol stays complete, and the status word reports it
+    if (threadIdx.x == 0 && chunk == 0 && p.status) atomicOr(p.status, 4);
+    src = 0;
+  }
   const uint32_t traj = (uint32_t)p.traj_id[row];
 
   const float4* __restrict__ xin = reinterpret_cast<const float4*>(p.x_in) + (size_t)src * p.quads_per_row;
@@ -197,10 +205,12 @@ static void dispatch_step(const StepParams& p, bool noise, bool unit_cx, dim3 gr
 int launch_step(int n_rows, int elems, int vel_dtype, const float* x_in, const void* vel,
                 const int32_t* src_rows, const int32_t* traj_id, float* x_out, float* logp_out,
                 uint64_t seed, int32_t step, double c_x, double c_v, double noise_std,
-                int logp_mean, RowScratch scratch, cudaStream_t stream) {
+                int logp_mean, RowScratch scratch, cudaStream_t stream, int rows_in, int32_t* status) {
   if (n_rows == 0) return PG_OK;
   const RowGeometry geo = row_geometry(n_rows, elems);
   StepParams p;
+  p.status = status;
+  p.rows_in = rows_in > 0 ? rows_in : n_rows;
   p.x_in = x_in;
   p.vel = vel;
   p.src_rows = src_rows;

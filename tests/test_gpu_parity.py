@@ -627,3 +627,48 @@ def test_native_rollout_and_graph_replay_equal_the_stepwise_driver(B):
         check(nat.replay())
     assert B.rollout_status(ro.h) == (w.n_groups * w.final_keep, w.n_steps, 0)
     ro.close()
+
+
+def test_out_of_range_gather_indices_are_reported_not_dereferenced(B):
+    G, N0, k, d = 2, 8, 4, 8192 + 64
+    h, _ = _handle(B, G, N0, d, T=3, stages=[(0, k)], seed=4)
+    try:
+        x = torch.randn(G * N0, d, device="cuda")
+        sc = torch.randn(G * N0, device="cuda")
+        keep = torch.empty(G * k, dtype=torch.int32, device="cuda")
+        src = torch.empty(G * k, dtype=torch.int32, device="cuda")
+        B.prune_ovf(h, 0, sc, keep, src)
+        good_src = src.clone()
+        bad = src.clone()
+        bad[1] = 10 ** 6
+        bad[5] = -1
+        y_bad = torch.zeros(G * k, d, device="cuda")
+        y_good = torch.zeros(G * k, d, device="cuda")
+        lp = torch.empty(G * k, device="cuda")
+        B.step(h, 0, (1.0, 0.1, 0.2), x, x, bad, y_bad, lp)
+        n_active, next_step, status = B.rollout_status(h, raise_on_flags=False)
+        assert status & 4 and next_step == 1
+        with pytest.raises(B.PgError) as e:
+            B.rollout_status(h)
+        assert e.value.code == B.EINDEX
+        # the rows with valid indices are unaffected (same noise: same trajectory ids and step)
+        B.rollout_reset(h)
+        B.prune_ovf(h, 0, sc, keep, src)
+        B.step(h, 0, (1.0, 0.1, 0.2), x, x, good_src, y_good, lp)
+        ok_rows = [i for i in range(G * k) if i not in (1, 5)]
+        assert torch.equal(y_bad[ok_rows], y_good[ok_rows])
+        assert B.rollout_status(h)[2] == 0
+        # compaction: a bad slot is skipped and reported
+        bad_keep = keep.clone()
+        bad_keep[2] = N0 + 3
+        dst = torch.full((G * k, d), -7.0, device="cuda")
+        B.compact(h, bad_keep, x, dst, d * 4)
+        assert B.rollout_status(h, raise_on_flags=False)[2] & 4
+        assert torch.all(dst[2] == -7.0) and torch.equal(dst[0], x[int(keep[0])])
+        narrow = torch.full((G * k,), -1, dtype=torch.int32, device="cuda")
+        B.compact(h, bad_keep, torch.arange(G * N0, dtype=torch.int32, device="cuda"), narrow, 4)
+        torch.cuda.synchronize()
+        assert int(narrow[2]) == -1 and int(narrow[0]) == int(keep[0])
+    finally:
+        torch.cuda.synchronize()
+        B.rollout_destroy(h)
