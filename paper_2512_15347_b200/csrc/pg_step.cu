@@ -270,26 +270,28 @@ int launch_philox_raw(int64_t n, const uint32_t* ctr, const uint32_t* key, uint3
 }
 
 __global__ void normal_rows_kernel(const __grid_constant__ PhiloxKeys rk, uint32_t step,
-                                   uint32_t stream_id, int quads_per_row, const int32_t* traj_id,
-                                   float* out) {
-  const int row = blockIdx.y;
-  const int q = blockIdx.x * blockDim.x + threadIdx.x;
-  if (q >= quads_per_row) return;
+                                   uint32_t stream_id, int quads_per_row, long long total_quads,
+                                   const int32_t* traj_id, float* out) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= total_quads) return;
+  const int row = (int)(i / quads_per_row);
+  const int q = (int)(i - (long long)row * quads_per_row);
   const uint4 r = philox4x32_10((uint32_t)q, step, (uint32_t)traj_id[row], stream_id, rk);
   float4 n;
   normal_pair(r.x, r.y, n.x, n.y);
   normal_pair(r.z, r.w, n.z, n.w);
-  reinterpret_cast<float4*>(out)[(size_t)row * quads_per_row + q] = n;
+  reinterpret_cast<float4*>(out)[i] = n;
 }
 
 int launch_normal_rows(uint64_t seed, int32_t step, int32_t stream_id, int n_rows, int d,
                        const int32_t* traj_id, float* out, cudaStream_t stream) {
   if (n_rows == 0) return PG_OK;
-  if (n_rows > 65535) return PG_EINVAL;
   const int quads = d / 4;
-  const dim3 grid((quads + 255) / 256, n_rows);
-  normal_rows_kernel<<<grid, 256, 0, stream>>>(make_philox_keys(seed), (uint32_t)step,
-                                               (uint32_t)stream_id, quads, traj_id, out);
+  const long long total = (long long)n_rows * quads;
+  const long long blocks = (total + 255) / 256;
+  if (blocks > 0x7FFFFFFFLL) return PG_EINVAL;
+  normal_rows_kernel<<<(unsigned)blocks, 256, 0, stream>>>(make_philox_keys(seed), (uint32_t)step,
+                                                           (uint32_t)stream_id, quads, total, traj_id, out);
   PG_LAUNCH_CHECK();
   return PG_OK;
 }

@@ -26,6 +26,19 @@ class RolloutOutput:
     std: Optional[torch.Tensor] = None
 
 
+def initial_latents(seed: int, n_groups: int, n_expand: int, elems: int, group_offset: int = 0,
+                    device=None) -> torch.Tensor:
+    """x_0 ~ N(0, I) for G * N0 trajectories from the library's counter-based generator (noise
+    stream 1, keyed by the global trajectory id), so any sharding of the groups draws the same
+    latents.  fp32 [G * N0, d]."""
+    dev = device or torch.device("cuda", torch.cuda.current_device())
+    rows = n_groups * n_expand
+    ids = torch.arange(group_offset * n_expand, group_offset * n_expand + rows, device=dev, dtype=torch.int32)
+    out = torch.empty(rows, elems, device=dev, dtype=torch.float32)
+    B.normal_rows(seed, 0, 1, rows, elems, ids, out)
+    return out
+
+
 class Rollout:
     """One Expand-and-Prune batch on the current CUDA device."""
 

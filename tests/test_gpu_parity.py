@@ -672,3 +672,23 @@ def test_out_of_range_gather_indices_are_reported_not_dereferenced(B):
     finally:
         torch.cuda.synchronize()
         B.rollout_destroy(h)
+
+
+def test_initial_latents_from_the_library_generator(B):
+    from paper_2512_15347_b200.rollout import initial_latents
+    G, N0, d = 3, 5, 4096
+    x = initial_latents(17, G, N0, d, group_offset=2).cpu().numpy()
+    for row in (0, 7, 14):
+        ref = oracle.normal_row(17, 0, 2 * N0 + row, d, stream=1)
+        assert np.abs(x[row] - ref).max() <= 3e-6
+    # a shard draws the rows of the whole batch
+    whole = initial_latents(17, 5, N0, d).cpu().numpy()
+    np.testing.assert_array_equal(x, whole[2 * N0:])
+    # stream 1 differs from the SDE noise stream of step 0
+    assert np.abs(x[0] - oracle.normal_row(17, 0, 2 * N0, d, stream=0)).max() > 1.0
+    assert abs(x.mean()) < 0.02 and abs(x.std() - 1.0) < 0.02
+    # many rows (more than one grid dimension used to allow)
+    ids = torch.arange(70000, dtype=torch.int32, device="cuda")
+    out = torch.empty(70000, 4, device="cuda")
+    B.normal_rows(1, 0, 1, 70000, 4, ids, out)
+    np.testing.assert_allclose(out[69999].cpu().numpy(), oracle.normal_row(1, 0, 69999, 4, stream=1), atol=3e-6)
