@@ -137,5 +137,10 @@ def compare_rollouts(w: wl.Workload, ref, out):
     e = latent_err(out.x_final.cpu().numpy(), ref.x_final)
     assert e <= LATENT_TOL, e
     k = w.final_keep
-    np.testing.assert_allclose(out.adv.cpu().numpy().reshape(w.n_groups, k), ref.adv, rtol=2e-4, atol=2e-5)
+    # rewards agree like scores; the advantages are the oracle's for the device's own rewards
+    # (they are ill-conditioned in the rewards when a group's spread is close to eps)
+    got_rw = out.rewards.cpu().numpy().reshape(w.n_groups, k)
+    assert np.abs(got_rw.astype(np.float64) - ref.rewards.astype(np.float64)).max() <= SCORE_GAP
+    adv_again, _, _ = oracle.advantages(got_rw, w.adv_eps)
+    np.testing.assert_allclose(out.adv.cpu().numpy().reshape(w.n_groups, k), adv_again, rtol=1e-5, atol=1e-6)
     return worst_lp, e
