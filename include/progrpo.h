@@ -107,6 +107,17 @@ int pg_rollout_destroy(pg_rollout *h);
 int pg_rollout_reset(pg_rollout *h, void *stream);
 
 /*
+ * Resume from a checkpoint.  The state of a rollout is (latents, next step, stages done,
+ * trajectory ids of the active rows, seed); noise is a pure function of (seed, trajectory id,
+ * step, element), so a handle restored to that state continues exactly as the interrupted run
+ * would have.  traj_ids: device [G * K] int32 with K the survivor count after `stages_done`
+ * stages (as returned by pg_rollout_traj_ids at checkpoint time).  The cursor must be reachable:
+ * all stages scheduled before next_step done, none scheduled after it (else PG_ESTATE).
+ */
+int pg_rollout_restore(pg_rollout *h, int32_t next_step, int32_t stages_done, const int32_t *traj_ids,
+                       void *stream);
+
+/*
  * Synchronises the device and reports the host-side cursor (trajectories
  * active in total, next step index) and the device status word (bit 0:
  * non-finite score seen by pg_prune_ovf, bit 1: a bounded wait expired, bit 2:

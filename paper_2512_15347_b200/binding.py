@@ -70,6 +70,7 @@ def lib() -> ctypes.CDLL:
     L.pg_rollout_init.argtypes = [ctypes.POINTER(Config), ctypes.POINTER(vp)]
     L.pg_rollout_destroy.argtypes = [vp]
     L.pg_rollout_reset.argtypes = [vp, vp]
+    L.pg_rollout_restore.argtypes = [vp, i32, i32, vp, vp]
     L.pg_rollout_status.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
     L.pg_step.argtypes = [vp, i32, ctypes.POINTER(StepCoef), vp, vp, vp, vp, vp, vp]
     L.pg_score.argtypes = [vp, ctypes.POINTER(PreviewCoef), vp, vp, vp, vp, vp]
@@ -105,7 +106,7 @@ def lib() -> ctypes.CDLL:
                  "pg_step", "pg_score", "pg_prune_ovf", "pg_compact", "pg_advantages",
                  "pg_ovf_select_batched", "pg_rollout_host", "pg_rollout_traj_ids",
                  "pg_philox_raw", "pg_normal_rows", "pg_score_static", "pg_policy_logprob",
-                 "pg_policy_objective", "pg_policy_backward", "pg_prune_uniform", "pg_group_stats", "pg_preview", "pg_rollout_run"):
+                 "pg_policy_objective", "pg_policy_backward", "pg_prune_uniform", "pg_group_stats", "pg_preview", "pg_rollout_run", "pg_rollout_restore"):
         getattr(L, name).restype = ctypes.c_int
     _lib = L
     return L
@@ -161,6 +162,11 @@ def rollout_destroy(h: int) -> None:
 
 def rollout_reset(h: int, stream=None) -> None:
     _check(lib().pg_rollout_reset(h, _stream(stream)), "pg_rollout_reset")
+
+
+def rollout_restore(h: int, next_step: int, stages_done: int, traj_ids, stream=None) -> None:
+    _check(lib().pg_rollout_restore(h, next_step, stages_done, _p(traj_ids), _stream(stream)),
+           "pg_rollout_restore")
 
 
 def rollout_status(h: int, raise_on_flags: bool = True):

@@ -133,6 +133,35 @@ int pg_rollout_reset(pg_rollout* h, void* stream) {
   return pg::launch_iota(h->d_traj[0], rows, h->cfg.group_offset * h->cfg.n_expand, st);
 }
 
+int pg_rollout_restore(pg_rollout* h, int32_t next_step, int32_t stages_done, const int32_t* traj_ids,
+                       void* stream) {
+  if (!h || !traj_ids) return PG_EINVAL;
+  if (next_step < 0 || next_step > h->cfg.n_steps || stages_done < 0 || stages_done > h->cfg.n_stages)
+    return PG_EINVAL;
+  // the cursor must be one the schedule can reach: every stage before next_step is done, and the
+  // stage scheduled at next_step itself may or may not have been pruned yet
+  for (int i = 0; i < h->cfg.n_stages; ++i) {
+    const bool done = i < stages_done;
+    if (h->stage_step[i] < next_step && !done) return PG_ESTATE;
+    if (h->stage_step[i] > next_step && done) return PG_ESTATE;
+  }
+  const int k_cur = stages_done > 0 ? h->stage_keep[stages_done - 1] : h->cfg.n_expand;
+  const int k_prev = stages_done > 1 ? h->stage_keep[stages_done - 2]
+                                     : (stages_done == 1 ? h->cfg.n_expand : 0);
+  cudaStream_t st = (cudaStream_t)stream;
+  PG_CUDA(cudaMemcpyAsync(h->d_traj[0], traj_ids, (size_t)h->cfg.n_groups * k_cur * sizeof(int32_t),
+                          cudaMemcpyDeviceToDevice, st));
+  PG_CUDA(cudaMemsetAsync(h->d_status, 0, sizeof(int32_t), st));
+  PG_CUDA(cudaMemsetAsync(h->d_tickets, 0,
+                          (size_t)h->cfg.n_groups * h->cfg.n_expand * sizeof(unsigned int), st));
+  h->traj_cur = 0;
+  h->next_step = next_step;
+  h->stage_cur = stages_done;
+  h->k_cur = k_cur;
+  h->k_prev = k_prev;
+  return PG_OK;
+}
+
 int pg_rollout_status(pg_rollout* h, int32_t* n_active, int32_t* next_step, int32_t* device_status) {
   if (!h) return PG_EINVAL;
   PG_CUDA(cudaDeviceSynchronize());

@@ -692,3 +692,54 @@ def test_initial_latents_from_the_library_generator(B):
     out = torch.empty(70000, 4, device="cuda")
     B.normal_rows(1, 0, 1, 70000, 4, ids, out)
     np.testing.assert_allclose(out[69999].cpu().numpy(), oracle.normal_row(1, 0, 69999, 4, stream=1), atol=3e-6)
+
+
+def test_checkpoint_restore_continues_bit_for_bit(B):
+    """Save (latents, cursor, trajectory ids) after a prune, restore them into a fresh handle and
+    finish the schedule: identical to the uninterrupted run."""
+    G, N0, d, T = 3, 10, 8192 + 128, 6
+    stages = [(1, 6), (4, 2)]
+    x0 = torch.randn(G * N0, d, device="cuda")
+    vels = [torch.randn(G * N0, d, device="cuda") for _ in range(T)]
+    scores = [torch.randn(G * N0, device="cuda") for _ in stages]
+
+    def run(h, x, start, stages_done, stop):
+        lp = torch.empty(G * N0, device="cuda")
+        k = N0 if stages_done == 0 else stages[stages_done - 1][1]
+        si = stages_done
+        for s in range(start, stop):
+            src = None
+            if si < len(stages) and stages[si][0] == s:
+                k_new = stages[si][1]
+                keep = torch.empty(G * k_new, dtype=torch.int32, device="cuda")
+                src = torch.empty(G * k_new, dtype=torch.int32, device="cuda")
+                B.prune_ovf(h, si, scores[si][: G * k], keep, src)
+                k, si = k_new, si + 1
+            y = torch.empty(G * k, d, device="cuda")
+            B.step(h, s, (1.0, 0.1, 0.3), x, vels[s], src, y, lp[: G * k])
+            x = y
+        return x, lp[: G * k].clone(), si
+
+    h, _ = _handle(B, G, N0, d, T=T, stages=stages, seed=31)
+    full_x, full_lp, _ = run(h, x0, 0, 0, T)
+    torch.cuda.synchronize()
+    B.rollout_destroy(h)
+
+    h, _ = _handle(B, G, N0, d, T=T, stages=stages, seed=31)
+    mid_x, _, done = run(h, x0, 0, 0, 3)                  # stops after step 2 (first prune done)
+    ids = torch.empty(G * 6, dtype=torch.int32, device="cuda")
+    B.rollout_traj_ids(h, ids)
+    saved = (mid_x.clone(), ids.clone(), 3, done)
+    torch.cuda.synchronize()
+    B.rollout_destroy(h)
+
+    h, _ = _handle(B, G, N0, d, T=T, stages=stages, seed=31)
+    with pytest.raises(B.PgError) as e:
+        B.rollout_restore(h, 3, 0, saved[1])                # stage at step 1 cannot be pending at step 3
+    assert e.value.code == B.ESTATE
+    B.rollout_restore(h, saved[2], saved[3], saved[1])
+    assert B.rollout_status(h) == (G * 6, 3, 0)
+    x, lp, _ = run(h, saved[0], 3, saved[3], T)
+    torch.cuda.synchronize()
+    assert torch.equal(x, full_x) and torch.equal(lp, full_lp)
+    B.rollout_destroy(h)
