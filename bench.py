@@ -206,6 +206,11 @@ def run_ours(args):
     if world > 1 or "TORCHELASTIC_RUN_ID" in os.environ:      # launched by torch.distributed.run
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        from paper_2512_15347_b200 import build as pg_build
+        pg_build.build()                 # no-op when libprogrpo.so is up to date; raises if nvcc fails
+    if dist is not None:
+        dist.barrier()
     B.lib()
     dev = torch.device("cuda", local)
     from dataclasses import replace

@@ -29,3 +29,13 @@ def pytest_collection_modifyitems(config, items):
 @pytest.fixture(scope="session")
 def golden_dir():
     return os.path.join(ROOT, "tests", "golden")
+
+
+@pytest.fixture(scope="session", autouse=True)
+def built_libraries():
+    """Builds the CUDA library (nvcc, no GPU needed) and the C oracle (gcc) when they are missing
+    or older than their sources, so that a fresh checkout can run the suite directly."""
+    from paper_2512_15347_b200 import build as pg_build
+    pg_build.build()
+    import oracle
+    oracle.build()
