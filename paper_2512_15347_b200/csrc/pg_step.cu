@@ -1,13 +1,13 @@
 // Fused Euler-Maruyama step + Gaussian policy log-probability (Eq. "euler_method").
 //
 // One CTA streams one chunk of one trajectory: x and the prediction are read once with
-// 128/64-bit coalesced loads (the loads of the next pair of quads are issued before the
-// current pair is computed; full chunks alternate between two register sets without bounds
-// checks), the noise is generated in registers (one Philox block per 4
-// elements), x' is written once.  Sum of squared noise: for a Box-Muller pair a^2 + b^2 equals
-// -2 ln u1, so the radius term is accumulated directly.  The per-trajectory sum is reduced
-// thread -> warp (shuffle) -> trajectory (fixed-slot partials finished by the last-arriving
-// warp, no barrier and no waiting), so the result does not depend on scheduling.
+// 128/64-bit coalesced loads, the loads of the next pair of quads being issued before the
+// current pair is computed (full chunks alternate between two register sets without bounds
+// checks); the noise is generated in registers (one Philox block per 4 elements); x' is written
+// once.  Sum of squared noise: for a Box-Muller pair a^2 + b^2 equals -2 ln u1, so the radius
+// term is accumulated directly.  The per-trajectory sum is reduced thread -> warp (shuffle) ->
+// CTA (shared memory) -> trajectory (fixed-slot partials finished by the last-arriving CTA,
+// without waiting), so the result does not depend on scheduling.
 #include "pg_common.cuh"
 
 namespace pg {
