@@ -59,8 +59,12 @@ template <> struct VelReg<__nv_bfloat16> { using type = VelBf16; };
 #define PG_STEP_UNROLL 2       // quads per thread and loop iteration (the next batch is in flight)
 #endif
 #ifndef PG_STEP_MIN_CTAS
-#define PG_STEP_MIN_CTAS 5     // __launch_bounds__ minimum resident CTAs per SM
+#define PG_STEP_MIN_CTAS 5     // __launch_bounds__ minimum resident CTAs per SM (bf16 prediction)
 #endif
+// fp32 predictions keep twice the prediction registers in flight: one CTA less per SM, no spills
+template <typename VelT, bool kNoise> struct StepMinCtas {
+  static constexpr int value = (sizeof(VelT) == 2 && kNoise) ? PG_STEP_MIN_CTAS : 4;
+};
 constexpr int kStepUnroll = PG_STEP_UNROLL;
 static_assert(kMinChunkQuads % (2 * kStepUnroll * kRowThreads) == 0 && kMaxChunkQuads % kMinChunkQuads == 0,
               "full chunks must hold an even number of batches");
@@ -99,7 +103,7 @@ __device__ __forceinline__ void step_quad(const StepParams& p, uint32_t traj, in
 
 // kNoise: noise_std > 0.  kUnitCx: c_x == 1 (drift = prediction), one FMA per element less.
 template <typename VelT, bool kNoise, bool kUnitCx>
-__global__ void __launch_bounds__(kRowThreads, PG_STEP_MIN_CTAS)
+__global__ void __launch_bounds__(kRowThreads, StepMinCtas<VelT, kNoise>::value)
 step_kernel(const __grid_constant__ StepParams p) {
   using VReg = typename VelReg<VelT>::type;
   const int row = blockIdx.x / p.chunks;
