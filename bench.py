@@ -34,7 +34,9 @@ if ROOT not in sys.path:
 # until the counters are taken again.
 STEP_KERNEL_TRAFFIC_RATIO = 0.984
 
-METRIC = "latent-steps/s (SDE step+logprob+OVF prune)"
+# the headline metric has three components: `value` is the first (latent-steps/s), the achieved HBM
+# GB/s is in `roofline` / `hbm_gbs_whole_rollout` / `prune_stage_gbs`, OVF groups/s in `ovf_microbench`
+METRIC = "latent-steps/s & achieved HBM GB/s (SDE step+logprob+OVF prune); OVF groups/s"
 UNIT = "latent-steps/s"
 
 
