@@ -119,28 +119,53 @@ def run_gpu(w: wl.Workload, inp: SharedInputs, record_scores=True):
 
 
 def compare_rollouts(w: wl.Workload, ref, out):
-    """Element-by-element comparison of a GPU rollout with the oracle's."""
-    for i, (s, k) in enumerate(w.stages):
-        got_keep = out.stage_keep[i].cpu().numpy().reshape(w.n_groups, k)
-        if out.stage_scores:
-            got_sc = out.stage_scores[i].cpu().numpy().reshape(ref.stage_scores[i].shape)
-            assert np.abs(got_sc.astype(np.float64) - ref.stage_scores[i].astype(np.float64)).max() <= SCORE_GAP
-            # given the device's own scores the selection must be the oracle's, bit for bit
-            keep_again, _ = oracle.ovf_select(got_sc, k)
-            np.testing.assert_array_equal(got_keep, keep_again)
-        np.testing.assert_array_equal(got_keep, ref.stage_keep[i])
-    np.testing.assert_array_equal(out.traj_id.cpu().numpy(), ref.traj_id)
+    """Element-by-element comparison of a GPU rollout with the oracle's.
+
+    Scores agree within SCORE_GAP, and given the device's own scores the selection is the oracle's
+    bit for bit.  Where the two selections nevertheless differ in a group, the difference can only
+    come from a score gap below that tolerance; the group is then two equally valid rollouts that
+    follow different trajectories, and it is left out of the later comparisons.  Returns
+    (worst log-prob error, latent error)."""
+    G = w.n_groups
+    same = np.ones(G, dtype=bool)          # groups whose survivors are still the oracle's
+    same_at_step = {}
+    stage_of = {s: i for i, (s, _) in enumerate(w.stages)}
+    for s in range(w.n_steps):
+        if s in stage_of:
+            i = stage_of[s]
+            k = w.stages[i][1]
+            got_keep = out.stage_keep[i].cpu().numpy().reshape(G, k)
+            if out.stage_scores:
+                got_sc = out.stage_scores[i].cpu().numpy().reshape(ref.stage_scores[i].shape)
+                diff = np.abs(got_sc.astype(np.float64) - ref.stage_scores[i].astype(np.float64))
+                assert diff[same].max(initial=0.0) <= SCORE_GAP
+                keep_again, _ = oracle.ovf_select(got_sc, k)
+                np.testing.assert_array_equal(got_keep, keep_again)
+                flipped = same & np.any(got_keep != ref.stage_keep[i], axis=1)
+                same &= ~flipped               # explained by a gap below the tolerance (asserted above)
+            else:
+                np.testing.assert_array_equal(got_keep[same], ref.stage_keep[i][same])
+        same_at_step[s] = same.copy()
+    if G >= 10:
+        assert same.mean() >= 0.9, "too many groups diverged for near-ties to explain"
+
+    def rows(mask, per):
+        return np.repeat(mask, per)
+
     worst_lp = 0.0
     for s in range(w.n_steps):
-        worst_lp = max(worst_lp, logp_err(out.logp[s].cpu().numpy(), ref.logp[s], w.elems))
+        m = rows(same_at_step[s], w.active_at(s))
+        worst_lp = max(worst_lp, logp_err(out.logp[s].cpu().numpy()[m], ref.logp[s][m], w.elems))
     assert worst_lp <= LOGP_TOL, worst_lp
-    e = latent_err(out.x_final.cpu().numpy(), ref.x_final)
-    assert e <= LATENT_TOL, e
     k = w.final_keep
+    m = rows(same, k)
+    np.testing.assert_array_equal(out.traj_id.cpu().numpy()[m], ref.traj_id[m])
+    e = latent_err(out.x_final.cpu().numpy()[m], ref.x_final[m])
+    assert e <= LATENT_TOL, e
     # rewards agree like scores; the advantages are the oracle's for the device's own rewards
     # (they are ill-conditioned in the rewards when a group's spread is close to eps)
-    got_rw = out.rewards.cpu().numpy().reshape(w.n_groups, k)
-    assert np.abs(got_rw.astype(np.float64) - ref.rewards.astype(np.float64)).max() <= SCORE_GAP
+    got_rw = out.rewards.cpu().numpy().reshape(G, k)
+    assert np.abs(got_rw.astype(np.float64) - ref.rewards.astype(np.float64))[same].max(initial=0.0) <= SCORE_GAP
     adv_again, _, _ = oracle.advantages(got_rw, w.adv_eps)
-    np.testing.assert_allclose(out.adv.cpu().numpy().reshape(w.n_groups, k), adv_again, rtol=1e-5, atol=1e-6)
+    np.testing.assert_allclose(out.adv.cpu().numpy().reshape(G, k), adv_again, rtol=1e-5, atol=1e-6)
     return worst_lp, e
