@@ -119,12 +119,17 @@ class Rollout:
             velocity: Callable[[int, torch.Tensor], torch.Tensor],
             external_scores: Optional[Callable[[int], torch.Tensor]] = None,
             final_rewards: Optional[Callable[[], torch.Tensor]] = None,
-            record_scores: bool = False, trace: Optional[list] = None) -> RolloutOutput:
+            record_scores: bool = False, trace: Optional[list] = None,
+            selector: str = "ovf") -> RolloutOutput:
         """Runs the whole schedule.  ``velocity(step, x_active)`` returns the prediction for the
         currently active rows; ``external_scores(stage)`` / ``final_rewards()`` return device
         fp32 tensors when the scores come from outside (else the preview mean / latent mean).
         x0 is only read (step 0 writes into the driver's own buffer).  With ``trace`` (a list),
-        every library call is bracketed by CUDA events: (kind, rows, start, end) is appended."""
+        every library call is bracketed by CUDA events: (kind, rows, start, end) is appended.
+        ``selector`` is "ovf" (Optimal Variance Filtering) or "uniform" (the random-subset
+        baseline; scores are then neither computed nor needed)."""
+        if selector not in ("ovf", "uniform"):
+            raise ValueError("selector must be 'ovf' or 'uniform'")
         self.reset()
         self.trace = trace
         out = RolloutOutput(x_final=None, logp=[], traj_id=None)
@@ -133,7 +138,13 @@ class Rollout:
         for s in range(self.T):
             vel = velocity(s, x_cur[: self.n_active])
             src = None
-            if stage_i < len(self.stages) and self.stages[stage_i][0] == s:
+            if stage_i < len(self.stages) and self.stages[stage_i][0] == s and selector == "uniform":
+                self._timed("prune", self.n_active, lambda: B.prune_uniform(
+                    self.h, stage_i, self.keep[stage_i], self.src_rows))
+                self.k_cur = self.stages[stage_i][1]
+                src = self.src_rows
+                stage_i += 1
+            elif stage_i < len(self.stages) and self.stages[stage_i][0] == s:
                 if external_scores is not None:
                     sc = external_scores(stage_i)
                 else:

@@ -743,3 +743,35 @@ def test_checkpoint_restore_continues_bit_for_bit(B):
     torch.cuda.synchronize()
     assert torch.equal(x, full_x) and torch.equal(lp, full_lp)
     B.rollout_destroy(h)
+
+
+def test_ovf_survivors_are_more_spread_out_than_uniform_survivors(B):
+    """The effect the method is built on (Fig. 2a): with reward-clustered scores, the survivors
+    chosen by OVF have a larger reward spread than a uniformly drawn subset of the same size -
+    measured end to end on the device with the library's own diagnostics."""
+    from paper_2512_15347_b200.rollout import Rollout
+    w = wl.scaled(wl.WORKLOADS["sd3"], n_groups=64, elems=256)
+    inp = U.SharedInputs(w)
+    table = {i: U.to_dev(wl.clustered_scores(w.n_groups, w.n_expand, w.seed, i, cluster_sigma=0.05,
+                                               outlier_frac=0.15, outlier_scale=0.3, nu=3.0).reshape(-1))
+             for i in (0, 1, 99)}
+    spread = {}
+    for selector in ("ovf", "uniform"):
+        ro = Rollout(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, torch.bfloat16)
+
+        def lookup(i):
+            ids = torch.empty(ro.n_active, device="cuda", dtype=torch.int32)
+            B.rollout_traj_ids(ro.h, ids)
+            return table[i][ids.long()]
+        # rewards of the survivors = the stage-1 score table (the quantity the last prune saw)
+        out = ro.run(U.to_dev(inp.x0), w.step_coef, w.preview_coef, lambda s, x: inp.vel_device(s, x),
+                     external_scores=lookup, final_rewards=lambda: lookup(1), selector=selector)
+        std = torch.empty(w.n_groups, device="cuda")
+        frac = torch.empty(w.n_groups, device="cuda")
+        B.group_stats(w.n_groups, w.final_keep, out.rewards, 0.5, None, std, frac)
+        torch.cuda.synchronize()
+        spread[selector] = (float(std.mean()), float(frac.mean()))
+        assert B.rollout_status(ro.h)[0] == w.n_groups * w.final_keep
+        ro.close()
+    assert spread["ovf"][0] > 1.3 * spread["uniform"][0]       # larger sigma_G
+    assert spread["ovf"][1] < spread["uniform"][1]             # fewer members clustered near the mean
