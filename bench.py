@@ -458,27 +458,38 @@ def run_e2e(B, wl, w, wr, rank, dist, dev, args):
     coefs = [w.step_coef(s) for s in range(w.n_steps)]
     pcoefs = [w.preview_coef(s) for s, _ in w.stages]
 
-    def call():
-        B.rollout_host(cfg, coefs, pcoefs, x0, vels, None, None, x_final, logp, keep, adv, ids, ws)
-
-    call()
-    torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
     n = max(1, min(args.steps, 3))
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record()
-    for _ in range(n):
+
+    def timed(x0_arg):
+        call = lambda: B.rollout_host(cfg, coefs, pcoefs, x0_arg, vels, None, None, x_final, logp, keep,
+                                      adv, ids, ws)
         call()
-    b.record()
-    torch.cuda.synchronize()
-    ms = sharding.max_over_ranks(a.elapsed_time(b), dist, dev)
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(n):
+            call()
+        b.record()
+        torch.cuda.synchronize()
+        return sharding.max_over_ranks(a.elapsed_time(b), dist, dev)
+
+    # headline: the initial latents are drawn on the device by the library's generator (x0 = NULL),
+    # so the host supplies only the per-step predictions; second figure: x0 copied from the host too
+    ms = timed(None)
+    ms_host_x0 = timed(x0)
     world = 1 if dist is None else dist.get_world_size()
-    h2d = x0.numel() * 4 + sum(v.numel() * v.element_size() for v in vels)
+    vel_bytes = sum(v.numel() * v.element_size() for v in vels)
     d2h = x_final.numel() * 4 + logp.numel() * 4 + keep.numel() * 4 + adv.numel() * 4 + ids.numel() * 4
-    return {"value": world * w.traj_steps * n / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+    return {"value": world * w.traj_steps * n / (ms * 1e-3), "unit": UNIT, "h2d_bytes_per_step": vel_bytes,
             "d2h_bytes_per_step": d2h, "ms_per_step": ms / n, "steps": n,
-            "entry": "pg_rollout_host (pinned host buffers, copies overlap compute)"}
+            "h2d_gbs": vel_bytes * n / (ms * 1e-3) / 1e9,
+            "entry": "pg_rollout_host (pinned host buffers; per-step predictions copied in while the previous "
+                     "step computes; x0 drawn on the device; latents, log-probs, indices, advantages copied out)",
+            "with_x0_from_host": {"value": world * w.traj_steps * n / (ms_host_x0 * 1e-3),
+                                  "ms_per_step": ms_host_x0 / n,
+                                  "h2d_bytes_per_step": vel_bytes + x0.numel() * 4}}
 
 
 def main():

@@ -284,7 +284,10 @@ int pg_ovf_select_batched(int32_t n_groups, int32_t n, int32_t k, const float *s
  * mean as score (or host-supplied scores), then the final reward stand-in
  * (mean of x_T, or host-supplied rewards) and the advantages, and copies the
  * results back.  Synchronises before returning.
- *   x0        host [G*N0, d] fp32
+ *   x0        host [G*N0, d] fp32, or NULL: the initial latents x_0 ~ N(0, I) of Section 5.1 are
+ *             then drawn on the device by the library's generator (the rows pg_normal_rows
+ *             gives for step 0, noise stream 1 and the global trajectory ids), so no latent
+ *             crosses the bus on the way in
  *   vel_steps host array of T pointers; vel_steps[s] is [rows_s, d] in
  *             cfg.vel_dtype with rows_s = rows alive when step s is predicted
  *             (G*K before any prune scheduled at s)

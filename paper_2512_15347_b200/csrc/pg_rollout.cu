@@ -420,7 +420,7 @@ int pg_rollout_host(const pg_config* cfg, const pg_step_coef* step_coef,
                     float* adv, int32_t* traj_id, void* workspace, size_t workspace_bytes) {
   int rc = validate_config(cfg);
   if (rc != PG_OK) return rc;
-  if (!step_coef || !x0 || !vel_steps || !workspace || !aligned16(workspace)) return PG_EINVAL;
+  if (!step_coef || !vel_steps || !workspace || !aligned16(workspace)) return PG_EINVAL;
   if (cfg->n_stages > 0 && !preview_coef && !stage_scores) return PG_EINVAL;
   const HostPlan pl = make_plan(cfg);
   if (workspace_bytes < pl.total) return PG_EINVAL;
@@ -483,7 +483,13 @@ int pg_rollout_host(const pg_config* cfg, const pg_step_coef* step_coef,
     return e;
   };
 
-  PG_TRY_CUDA(cudaMemcpyAsync(d_x[0], x0, pl.x_bytes, cudaMemcpyHostToDevice, compute));
+  if (x0) {
+    PG_TRY_CUDA(cudaMemcpyAsync(d_x[0], x0, pl.x_bytes, cudaMemcpyHostToDevice, compute));
+  } else {
+    // initial latents drawn on the device (noise stream 1, keyed by trajectory id): nothing to copy
+    PG_TRY(pg::launch_normal_rows(cfg->seed, 0, 1, (int)pl.rows0, cfg->elems, h->d_traj[h->traj_cur],
+                                  d_x[0], compute));
+  }
   PG_TRY_CUDA(prefetch(0));
   int cur = 0, stage = 0;
   size_t logp_off = 0, keep_off = 0;

@@ -392,6 +392,44 @@ def test_host_buffer_rollout_matches_device_rollout(B):
     ro.close()
 
 
+def test_host_buffer_rollout_draws_its_own_initial_latents(B):
+    """x0 = NULL: the library draws x_0 ~ N(0, I) on the device (noise stream 1).  The result is
+    the rollout that starts from those rows handed in as a host buffer, bit for bit, and the rows
+    themselves are the oracle's normals for that stream."""
+    from paper_2512_15347_b200.rollout import initial_latents
+    w = wl.scaled(wl.WORKLOADS["large"], n_groups=2, elems=8192 + 1024)
+    inp = U.SharedInputs(w)
+    offset = 3
+    cfg = B.make_config(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, B.VEL_BF16,
+                        adv_eps=w.adv_eps, group_offset=offset)
+    ws = torch.empty(B.rollout_host_workspace_bytes(cfg), dtype=torch.uint8, device="cuda")
+    x0_dev = initial_latents(w.seed, w.n_groups, w.n_expand, w.elems, group_offset=offset)
+    for row in (0, w.n_groups * w.n_expand - 1):
+        ref = oracle.normal_row(w.seed, 0, offset * w.n_expand + row, w.elems, stream=1)
+        assert np.abs(x0_dev[row].cpu().numpy() - ref).max() <= 3e-6
+    vels = []
+    for s in range(w.n_steps):
+        rows = w.n_groups * w.rows_before(s)
+        vels.append(U.vel_to_dev(inp.vel_numpy(s, np.empty((rows, 0)))).cpu().pin_memory())
+    K = w.final_keep
+    coefs = [w.step_coef(s) for s in range(w.n_steps)]
+    pcoefs = [w.preview_coef(s) for s, _ in w.stages]
+
+    def run(x0):
+        res = (torch.empty(w.n_groups * K, w.elems).pin_memory(), torch.empty(w.traj_steps).pin_memory(),
+               torch.empty(sum(w.n_groups * k for _, k in w.stages), dtype=torch.int32).pin_memory(),
+               torch.empty(w.n_groups * K).pin_memory(),
+               torch.empty(w.n_groups * K, dtype=torch.int32).pin_memory())
+        assert B.rollout_host(cfg, coefs, pcoefs, x0, vels, None, None, *res, ws) == 0
+        return res
+
+    drawn = run(None)
+    given = run(x0_dev.cpu().pin_memory())
+    for a, b in zip(drawn, given):
+        assert torch.equal(a, b)
+    assert torch.isfinite(drawn[0]).all() and drawn[4].min() >= offset * w.n_expand
+
+
 # ------------------------------------------------------------------ call-order and argument errors
 
 def test_out_of_sequence_calls_are_refused(B):
