@@ -2,10 +2,10 @@
 // (Eq. "advK"), clustering diagnostics and the uniform-subsampling baseline.
 //
 // Selection: one warp per group; the scores become order-preserving 32-bit keys, are sorted in
-// registers, every element finds its rank in the total order (score, slot), the running sums
-// from both ends give the k+1 candidate variances "j lowest + (k-j) highest" in fp64 with
-// explicitly rounded operations, and the kept slots are written in ascending slot order through
-// a popcount prefix sum.
+// registers, the running sums from both ends give the k+1 candidate variances "j lowest + (k-j)
+// highest" in fp64 with explicitly rounded operations, membership follows from the keys at the
+// two cuts (from ranks in the total order (score, slot) when keys tie there), and the kept slots
+// are written in ascending slot order through a popcount prefix sum.
 #include "pg_common.cuh"
 #include <float.h>
 
@@ -54,14 +54,17 @@ __device__ __forceinline__ double arithmetic_value(float s) {
 //  1. The 32-bit order keys alone are sorted with a bitonic network held in registers (one
 //     integer min and one max per compare-exchange; shuffles for distances of E and more).
 //     Slots >= n hold an all-ones key and sort to the end.
-//  2. Each element finds its rank in the total order (score, slot) by a binary search for its
-//     key in the sorted list; where equal keys exist (rare for real scores) the rank is advanced
-//     by the number of equal keys in lower slots, counted directly.  Ranks are a permutation.
-//  3. Running sums from both ends: the centred values and their squares are formed by all lanes
-//     in parallel, then lanes 0 and 1 accumulate them serially, in order, in fp64 with explicitly
-//     rounded operations - the same operations in the same order as a plain serial loop.
-//  4. k+1 candidates, argmax with the "largest j" tie rule, membership by rank; every lane holds
-//     its scores in slot order, so a popcount prefix over lanes gives ascending slot order.
+//  2. Running sums from both ends: the centred values and their squares are formed by all lanes
+//     in parallel, then lanes 0..3 accumulate one sequence each serially, in order, in fp64 with
+//     explicitly rounded operations - the same operations in the same order as a plain serial loop.
+//  3. k+1 candidates, argmax with the "largest j" tie rule.
+//  4. Membership: by comparison with the two keys at the cuts of the order; only when a key just
+//     inside a cut equals the one just outside it (rare for real scores) is the rank of every
+//     element in the total order (score, slot) worked out, by a binary search in the sorted keys
+//     plus a direct count of equal keys in lower slots.  Every lane holds its scores in slot
+//     order, so a popcount prefix over lanes gives ascending slot order.
+//  5. Kept scores go through shared memory so that their stores, the advantage statistics and
+//     the single division are spread over the lanes.
 // warps (= groups) per CTA: four while the per-warp shared memory allows it, one for wide groups
 template <int E> struct OvfWarps { static constexpr int value = (E <= 8) ? 4 : 1; };
 constexpr int kBulkWaitLimit = 1 << 14;   // mbarrier try_wait attempts before giving up
@@ -149,7 +152,6 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
       mine[r] = 0xFFFFFFFFu;
     }
     key[r] = mine[r];
-    okey[i] = mine[r];
   }
   if (bad && p.status) atomicOr(p.status, 1);
 
@@ -202,26 +204,6 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
   for (int r = 0; r < E; ++r) skey[lane * E + r] = key[r];
   __syncwarp();
 
-  // 2. rank of every own element in the order (score, slot)
-  int rank[E];
-#pragma unroll
-  for (int r = 0; r < E; ++r) {
-    int pos = 0;
-#pragma unroll
-    for (int step = N / 2; step > 0; step >>= 1)
-      if (skey[pos + step - 1] < mine[r]) pos += step;
-    rank[r] = pos;                                  // first position whose key is >= mine
-  }
-#pragma unroll
-  for (int r = 0; r < E; ++r) {
-    const int i = lane * E + r;
-    if (i < n && rank[r] + 1 < N && skey[rank[r] + 1] == mine[r]) {   // equal keys exist
-      int lower_slots = 0;
-      for (int j = 0; j < i; ++j) lower_slots += (okey[j] == mine[r]) ? 1 : 0;
-      rank[r] += lower_slots;
-    }
-  }
-
   // 3. centred values and squares in parallel, then the serial running sums
   const double pivot = arithmetic_value(key_to_score(skey[n / 2]));
   for (int j = lane; j < k; j += 32) {
@@ -233,17 +215,14 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
     H2[j + 1] = __dmul_rn(ch, ch);
   }
   __syncwarp();
-  if (lane < 2) {
-    double* S1 = lane == 0 ? L1 : H1;
-    double* S2 = lane == 0 ? L2 : H2;
-    double a1 = 0.0, a2 = 0.0;
-    S1[0] = 0.0;
-    S2[0] = 0.0;
+  if (lane < 4) {                       // L1, L2, H1, H2 are contiguous: one serial chain per lane
+    double* S = L1 + (size_t)lane * (k + 1);
+    double a = 0.0;
+    S[0] = 0.0;
+#pragma unroll 4
     for (int j = 1; j <= k; ++j) {
-      a1 = __dadd_rn(a1, S1[j]);
-      a2 = __dadd_rn(a2, S2[j]);
-      S1[j] = a1;
-      S2[j] = a2;
+      a = __dadd_rn(a, S[j]);
+      S[j] = a;
     }
   }
   __syncwarp();
@@ -269,10 +248,43 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
   const int high_from = n - (k - jstar);
   if (lane == 0 && p.sel_var) p.sel_var[g] = (float)(best_m / ((double)k * (double)k));
 
+  // 5. membership.  With distinct keys at both cuts of the order an element is kept exactly when
+  //    its key is at most the j*-th lowest or at least the (k - j*)-th highest key.  Only when the
+  //    key just inside a cut equals the key just outside it does the slot decide: then every
+  //    element finds its rank in the total order (score, slot) by a binary search for its key in
+  //    the sorted list, advanced by the number of equal keys in lower slots.
+  const int n_high = k - jstar;
+  const uint32_t lowkey = jstar > 0 ? skey[jstar - 1] : 0u;
+  const uint32_t highkey = n_high > 0 ? skey[high_from] : 0xFFFFFFFFu;
+  const bool cut_tie = (jstar > 0 && jstar < n && skey[jstar] == lowkey) ||
+                       (n_high > 0 && high_from > 0 && skey[high_from - 1] == highkey);
   unsigned int bits = 0u;
+  if (!cut_tie) {                                   // uniform over the warp
 #pragma unroll
-  for (int r = 0; r < E; ++r)
-    if (lane * E + r < n && (rank[r] < jstar || rank[r] >= high_from)) bits |= 1u << r;
+    for (int r = 0; r < E; ++r) {
+      const bool in_low = jstar > 0 && mine[r] <= lowkey;
+      const bool in_high = n_high > 0 && mine[r] >= highkey;
+      if (lane * E + r < n && (in_low || in_high)) bits |= 1u << r;
+    }
+  } else {
+#pragma unroll
+    for (int r = 0; r < E; ++r) okey[lane * E + r] = mine[r];
+    __syncwarp();
+#pragma unroll
+    for (int r = 0; r < E; ++r) {
+      const int i = lane * E + r;
+      int rank = 0;
+#pragma unroll
+      for (int step = N / 2; step > 0; step >>= 1)
+        if (skey[rank + step - 1] < mine[r]) rank += step;    // first position whose key is >= mine
+      if (i < n && rank + 1 < N && skey[rank + 1] == mine[r]) {  // equal keys exist
+        int lower_slots = 0;
+        for (int j = 0; j < i; ++j) lower_slots += (okey[j] == mine[r]) ? 1 : 0;
+        rank += lower_slots;
+      }
+      if (i < n && (rank < jstar || rank >= high_from)) bits |= 1u << r;
+    }
+  }
   const int cnt = __popc(bits);
   int incl = cnt;
 #pragma unroll
@@ -281,8 +293,10 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
     if (lane >= o) incl += t;
   }
   const int first = lane * E;
+  const bool want_scores = p.kept_scores || p.adv;
+  float* kept_s = reinterpret_cast<float*>(L1);     // [k], reuses the running sums' space
+  __syncwarp();                                     // every lane is done with the running sums
   int pos = incl - cnt;
-  double sum_kept = 0.0;
 #pragma unroll
   for (int r = 0; r < E; ++r) {
     if (bits & (1u << r)) {
@@ -291,28 +305,30 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
       p.keep_idx[o] = i;
       if (p.src_rows) p.src_rows[o] = g * n + i;
       if (p.traj_out) p.traj_out[o] = p.traj_in[(size_t)g * n + i];
-      if (p.kept_scores) p.kept_scores[o] = orig[r];
-      sum_kept += (double)orig[r];
+      if (want_scores) kept_s[pos] = orig[r];
       ++pos;
     }
   }
-  if (p.adv) {
-    const double mu = warp_sum(sum_kept) / (double)k;
-    double sq = 0.0;
-#pragma unroll
-    for (int r = 0; r < E; ++r)
-      if (bits & (1u << r)) {
-        const double dlt = (double)orig[r] - mu;
+  if (want_scores) {
+    // kept scores in slot order, now spread over the lanes: coalesced stores, one division
+    __syncwarp();
+    double sum_kept = 0.0;
+    for (int j = lane; j < k; j += 32) {
+      const float v = kept_s[j];
+      if (p.kept_scores) p.kept_scores[(size_t)g * k + j] = v;
+      sum_kept += (double)v;
+    }
+    if (p.adv) {
+      const double mu = warp_sum(sum_kept) / (double)k;
+      double sq = 0.0;
+      for (int j = lane; j < k; j += 32) {
+        const double dlt = (double)kept_s[j] - mu;
         sq += dlt * dlt;
       }
-    const double denom = sqrt(warp_sum(sq) / (double)k) + (double)p.adv_eps;
-    pos = incl - cnt;
-#pragma unroll
-    for (int r = 0; r < E; ++r)
-      if (bits & (1u << r)) {
-        p.adv[(size_t)g * k + pos] = (float)(((double)orig[r] - mu) / denom);
-        ++pos;
-      }
+      const double inv = 1.0 / (sqrt(warp_sum(sq) / (double)k) + (double)p.adv_eps);
+      for (int j = lane; j < k; j += 32)
+        p.adv[(size_t)g * k + j] = (float)(((double)kept_s[j] - mu) * inv);
+    }
   }
 }
 

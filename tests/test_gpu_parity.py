@@ -151,8 +151,11 @@ def _ovf_cases():
     for G, n, k in shapes:
         yield "normal", rng.standard_normal((G, n)).astype(np.float32), k
         yield "ties", rng.integers(0, 4, (G, n)).astype(np.float32), k
+        # a few equal scores among distinct ones: a tie sits at one cut of the order in some groups only
+        yield "sparse-ties", (np.round(rng.standard_normal((G, n)) * 8) / 8).astype(np.float32), k
         yield "clustered", wl.clustered_scores(G, n, seed=n + k, stage=0, cluster_sigma=0.05,
                                                outlier_frac=0.15, outlier_scale=0.3, nu=3.0), k
+    yield "coarse", np.round(rng.standard_normal((512, 32)), 1).astype(np.float32), 16
     yield "equal", np.full((3, 40), 1.25, np.float32), 7
     z = np.zeros((2, 8), np.float32)
     z[:, ::2] = -0.0
