@@ -352,6 +352,20 @@ def run_ours(args):
                            "pg_rollout_run, one call per rollout; graph = that call captured and replayed"}
         del nat
 
+    def timed(fn, reps=10):
+        """Median device time (ms) of one call, after three warm-up calls."""
+        ts = []
+        for i in range(reps + 3):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            if i >= 3:
+                ts.append(a.elapsed_time(b))
+        ts.sort()
+        return ts[len(ts) // 2]
+
     # policy-update kernels on the survivors' shape (secondary numbers; not part of `value`)
     policy = None
     if rank == 0 and w.vel_dtype == "bf16" and w.velocity == "normal":
@@ -364,18 +378,6 @@ def run_ours(args):
         grad = torch.empty(rows, w.elems, device=dev, dtype=torch.bfloat16)
         coef = w.step_coef(0)
 
-        def timed(fn, reps=10):
-            ts = []
-            for i in range(reps + 3):
-                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                a.record()
-                fn()
-                b.record()
-                torch.cuda.synchronize()
-                if i >= 3:
-                    ts.append(a.elapsed_time(b))
-            ts.sort()
-            return ts[len(ts) // 2]
         t_lp = timed(lambda: B.policy_logprob(ro.h, coef, xa, xb, va, vb, lp, klv))
         t_bw = timed(lambda: B.policy_backward(ro.h, coef, xa, xb, va, vb, dl, -1e-6, grad))
         policy = {"rows": rows, "logprob_kl_gbs": rows * w.elems * 12 / (t_lp * 1e-3) / 1e9,
@@ -383,6 +385,32 @@ def run_ours(args):
                   "bytes_per_element": {"logprob_kl": 12, "backward": 14},
                   "note": "per-step kernels of the update on the survivors (x, x_next fp32; new and "
                           "reference predictions bf16; bf16 gradient), inputs larger than L2"}
+
+    # physical compaction and preview emission on the first stage's shape (secondary numbers: the
+    # rollout folds the compaction into the next step's gather and scores without emitting)
+    other = None
+    if rank == 0 and w.vel_dtype == "bf16" and w.velocity == "normal" and w.stages:
+        k0 = w.stages[0][1]
+        rows_in, rows_out = w.n_groups * w.n_expand, w.n_groups * k0
+        hc = B.rollout_init(B.make_config(w.n_groups, w.n_expand, w.elems, 1, [(0, k0)], w.seed, B.VEL_BF16))
+        sc0 = torch.randn(rows_in, device=dev)
+        keep0 = torch.empty(rows_out, dtype=torch.int32, device=dev)
+        B.prune_ovf(hc, 0, sc0, keep0)
+        src_x, dst_x = ro.x[0][:rows_in], ro.x[1][:rows_out]
+        t_c = timed(lambda: B.compact(hc, keep0, src_x, dst_x, w.elems * 4))
+        B.rollout_destroy(hc)
+        hp = B.rollout_init(B.make_config(w.n_groups, k0, w.elems, 1, [], w.seed, B.VEL_BF16))
+        xs, vs = ro.x[0][:rows_out], vels[0][:rows_out]
+        out16 = torch.empty(rows_out, w.elems, device=dev, dtype=torch.bfloat16)
+        t_p16 = timed(lambda: B.preview(hp, (1.0, 0.5), xs, vs, out16))
+        del out16
+        B.rollout_destroy(hp)
+        other = {"compact_gbs": rows_out * w.elems * 8 / (t_c * 1e-3) / 1e9,
+                 "compact_rows": [rows_in, rows_out],
+                 "preview_bf16_gbs": rows_out * w.elems * 8 / (t_p16 * 1e-3) / 1e9,
+                 "bytes_per_element": {"compact": 8, "preview_bf16": 8},
+                 "note": "pg_compact gathers the first stage's survivors (fp32 rows); pg_preview writes "
+                         "the bf16 look-ahead latent for an external decoder"}
 
     # end to end through the host-buffer entry point (pinned host memory, copies inside the timing)
     e2e = None
@@ -410,7 +438,7 @@ def run_ours(args):
                                 v["launches"] // args.steps} for k, v in kinds.items()},
                 "score_gbs": score_gbs, "prune_stage_gbs": prune_stage_gbs,
                 "hbm_gbs_whole_rollout": (step_bytes + (score_bytes if score_gbs else 0)) / (total_ms * 1e-3) / 1e9,
-                "ovf_microbench": ovf, "drivers": drivers, "policy_update": policy, "e2e": e2e, "cpu_baseline": cpu_base}
+                "ovf_microbench": ovf, "drivers": drivers, "policy_update": policy, "other_kernels": other, "e2e": e2e, "cpu_baseline": cpu_base}
         print(json.dumps(line))
     ro.close()
     if dist is not None:

@@ -8,6 +8,11 @@ namespace pg {
 constexpr int kCompactThreads = 256;
 constexpr size_t kCompactPiece = 32768;   // bytes per CTA
 
+__device__ __forceinline__ uint4 ldcs_word(const uint4* p) { return __ldcs(p); }
+__device__ __forceinline__ void stcs_word(uint4* p, const uint4& v) { __stcs(p, v); }
+template <typename T> __device__ __forceinline__ T ldcs_word(const T* p) { return *p; }
+template <typename T> __device__ __forceinline__ void stcs_word(T* p, const T& v) { *p = v; }
+
 template <typename T>
 __global__ void __launch_bounds__(kCompactThreads)
 compact_kernel(const int32_t* keep_idx, const unsigned char* src, unsigned char* dst,
@@ -25,6 +30,18 @@ compact_kernel(const int32_t* keep_idx, const unsigned char* src, unsigned char*
   const T* s = reinterpret_cast<const T*>(src + ((size_t)g * n_prev + slot) * row_bytes + begin);
   T* d = reinterpret_cast<T*>(dst + (size_t)row * row_bytes + begin);
   const size_t count = (end - begin) / sizeof(T);
+  constexpr size_t kFull = kCompactPiece / sizeof(T);
+  constexpr int kPerThread = (int)(kFull / kCompactThreads);
+  if constexpr (sizeof(T) == 16) if (count == kFull) {
+    // full piece of 16-byte words: all loads of the thread in flight before the first store,
+    // streaming hints on both sides (every byte is touched once)
+    T r[kPerThread];
+#pragma unroll
+    for (int u = 0; u < kPerThread; ++u) r[u] = ldcs_word(s + threadIdx.x + u * kCompactThreads);
+#pragma unroll
+    for (int u = 0; u < kPerThread; ++u) stcs_word(d + threadIdx.x + u * kCompactThreads, r[u]);
+    return;
+  }
   for (size_t i = threadIdx.x; i < count; i += kCompactThreads) d[i] = s[i];
 }
 
