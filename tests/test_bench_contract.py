@@ -1,0 +1,63 @@
+"""bench.py prints one JSON line with the agreed keys: the CPU arm (the oracle, timed) is checked
+here without a GPU, the GPU arm on a small workload."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+BASE_KEYS = ("metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_step", "higher_is_better",
+             "scaling", "vs_baseline", "dtype", "data", "config", "e2e", "cpu_baseline", "gpu_launches")
+
+
+def _run(args, env_extra=None, timeout=600):
+    env = dict(os.environ)
+    env.update(env_extra or {})
+    p = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py")] + args, cwd=ROOT, env=env,
+                       capture_output=True, text=True, timeout=timeout)
+    assert p.returncode == 0, p.stderr[-2000:]
+    return [ln for ln in p.stdout.splitlines() if ln.strip()]
+
+
+def test_reference_arm_prints_one_line_with_the_contract_keys():
+    lines = _run(["--impl", "reference", "--workload", "sd15", "--steps", "1", "--warmup", "1"])
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    for k in BASE_KEYS:
+        assert k in d, k
+    assert d["impl"] == "reference" and d["unit"] == "latent-steps/s" and d["higher_is_better"] is True
+    assert d["value"] > 0 and d["steps"] == 1 and d["vs_baseline"] is None and d["dtype"] == "f64"
+    assert "workload" in d["config"] and d["config"]["workload"].startswith("sd15")
+    cb = d["cpu_baseline"]
+    assert cb["kind"] == "oracle" and cb["cores"] >= 1 and cb["sample"] and cb["value"] == d["value"]
+    e = d["e2e"]
+    assert e["value"] == d["value"] and e["unit"] == d["unit"]
+    assert e["h2d_bytes_per_step"] == 0 and e["d2h_bytes_per_step"] == 0
+    assert d["gpu_launches"] == 0
+
+
+def test_reference_arm_is_silent_on_other_ranks():
+    assert _run(["--impl", "reference", "--workload", "sd15", "--steps", "1", "--warmup", "1"],
+                {"RANK": "1", "WORLD_SIZE": "2", "LOCAL_RANK": "1"}) == []
+
+
+@pytest.mark.gpu
+def test_gpu_arm_prints_roofline_baseline_and_end_to_end():
+    lines = _run(["--workload", "sd15", "--steps", "3", "--warmup", "3"])
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    for k in BASE_KEYS + ("roofline", "clocks"):
+        assert k in d, k
+    assert "impl" not in d and d["n_gpus"] == 1 and d["warmup"] >= 3 and d["dtype"] == "f32"
+    assert d["value"] > 0 and d["gpu_launches"] > 0 and d["scaling"] == "weak"
+    r = d["roofline"]
+    assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["peak"] > 0 and r["achieved"] > 0
+    assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9 and "traffic" in r
+    cb = d["cpu_baseline"]
+    assert cb["kind"] == "oracle" and cb["value"] > 0 and cb["cores"] >= 1 and cb["sample"]
+    e = d["e2e"]
+    assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0
+    assert e["value"] != d["value"]
+    assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
