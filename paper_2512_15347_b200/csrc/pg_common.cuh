@@ -118,12 +118,13 @@ __device__ __forceinline__ double warp_sum(double v) {
 // ---------------------------------------------------------------- launch geometry
 // Row-streaming kernels (step, score): a CTA of kRowThreads threads handles one chunk of one
 // row and contributes one partial sum, so a row owns `chunks` partial slots.  Chunks are
-// 2048..8192 quads (4-element groups): short chunks pay the end-of-CTA reduction (a barrier, a
-// fence and an atomic) too often, long ones leave too few CTAs to fill 148 SMs evenly.
+// 2048 or 4096 quads (4-element groups): shorter chunks pay the end-of-CTA reduction (a barrier,
+// a fence and an atomic) too often, longer ones measured 1 % slower in back-to-back launches and
+// 4 % slower in isolated ones (fewer, longer CTAs drain less evenly at the end of a launch).
 constexpr int kRowThreads = 256;
 constexpr int kRowWarps = kRowThreads / 32;
 constexpr int kMinChunkQuads = 2048;                   // 8192 elements
-constexpr int kMaxChunkQuads = 8192;                   // 32768 elements
+constexpr int kMaxChunkQuads = 4096;                   // 16384 elements
 constexpr long long kWantedCtas = 148LL * 4 * 16;      // CTAs for ~16 waves at 4 CTAs per SM
 
 struct RowGeometry {

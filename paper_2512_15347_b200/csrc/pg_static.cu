@@ -21,6 +21,7 @@ namespace {
 constexpr int kStaticMaxRows = PG_STATIC_MAX_ROWS;
 constexpr size_t kStaticMaxPartials = PG_STATIC_MAX_PARTIALS;
 constexpr int kMaxDevices = 64;
+constexpr int kStaticChunkQuads = 8192;   // 32768 elements per partial sum: the limit the header documents
 
 struct StaticScratch {
   float partials[kStaticMaxPartials];
@@ -61,7 +62,7 @@ extern "C" int pg_score_static(int32_t n_rows, int32_t elems, int32_t vel_dtype,
   if (((uintptr_t)x & 15) || ((uintptr_t)vel & 15)) return PG_EINVAL;
   // capacity of the built-in scratch: PG_STATIC_MAX_ROWS rows, PG_STATIC_MAX_PARTIALS partial sums
   if (n_rows > kStaticMaxRows) return PG_ECAPACITY;
-  const pg::RowGeometry geo = pg::row_geometry(n_rows, elems, pg::kMaxChunkQuads);
+  const pg::RowGeometry geo = pg::row_geometry(n_rows, elems, kStaticChunkQuads);
   const size_t need = (size_t)n_rows * (size_t)geo.chunks;
   if (need > kStaticMaxPartials) return PG_ECAPACITY;
 
@@ -73,5 +74,5 @@ extern "C" int pg_score_static(int32_t n_rows, int32_t elems, int32_t vel_dtype,
   PG_CUDA(cudaMemsetAsync(s->tickets, 0, (size_t)n_rows * sizeof(unsigned int), st));
   pg::RowScratch scratch{s->partials, s->tickets};
   return pg::launch_score(n_rows, elems, vel_dtype, x, vel, coef->p_x, coef->p_v, scores_out,
-                          nullptr, scratch, st, pg::kMaxChunkQuads);
+                          nullptr, scratch, st, kStaticChunkQuads);
 }
