@@ -114,11 +114,21 @@ class OracleSample:
 
     def __init__(self, w, groups: int):
         from paper_2512_15347_b200 import workloads as wl
+        import torch
         self.w = w
-        self.sw = wl.scaled(w, n_groups=groups)
-        self.x0 = wl.initial_latents(self.sw).numpy()
-        self.vels = [wl.as_numpy_velocity(wl.normal_velocity(self.sw, s, groups * w.rows_before(s)))
-                     for s in range(w.n_steps)]
+        self.sw = sw = wl.scaled(w, n_groups=groups)
+        self.x0 = wl.initial_latents(sw).numpy()
+        if w.velocity == "affine":
+            a, b = wl.affine_field(sw)
+            self.velocity = lambda s, x, traj: wl.affine_velocity(torch.from_numpy(x), a, b).numpy()
+        else:
+            vels = [wl.as_numpy_velocity(wl.normal_velocity(sw, s, groups * w.rows_before(s)))
+                    for s in range(w.n_steps)]
+            self.velocity = lambda s, x, traj: vels[s]
+        self.ext = self.fin = None
+        if w.scores == "external":
+            self.ext = lambda stage, traj: wl.sd3_stage_scores(sw, stage, traj)
+            self.fin = lambda x, traj: wl.sd3_stage_scores(sw, 99, traj)
         self.desc = (f"first {groups} of {w.n_groups} prompt groups, full schedule, full-length latents "
                      f"({self.sw.traj_steps} of {w.traj_steps} latent-steps)")
 
@@ -128,11 +138,14 @@ class OracleSample:
         sw = self.sw
         t0 = time.perf_counter()
         oracle.rollout(self.x0, sw.n_groups, sw.n_expand, sw.n_steps, sw.stages, sw.seed, sw.step_coef,
-                       sw.preview_coef, lambda s, x, traj: self.vels[s], adv_eps=sw.adv_eps)
+                       sw.preview_coef, self.velocity, external_scores=self.ext, final_rewards=self.fin,
+                       adv_eps=sw.adv_eps)
         return time.perf_counter() - t0
 
 
 ORACLE_GROUPS = 8
+# smaller workloads reported beside the bench line: (name, prompt groups of the oracle's sample)
+OTHER_WORKLOADS = (('sd3', 4), ('sd15', 8), ('tiny', 1))
 
 
 def run_reference(args):
@@ -179,50 +192,16 @@ def _config(w, args):
 
 # ------------------------------------------------------------------ GPU arm
 
-def run_ours(args):
+def _gpu_inputs(w, wr, ro, dev, rank):
+    """Seeded device inputs of one workload: initial latents, the per-step predictions (or the
+    stand-in network for the affine field), and the stand-in reward model of the workloads whose
+    scores come from outside."""
     import torch
     from paper_2512_15347_b200 import binding as B
     from paper_2512_15347_b200 import workloads as wl
     from paper_2512_15347_b200 import sharding
-    from paper_2512_15347_b200.rollout import Rollout
-
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    w = wl.WORKLOADS[args.workload]
-    if args.groups:
-        w = wl.scaled(w, n_groups=args.groups, name=f"{w.name}[{args.groups} groups]")
-
-    cpu_base = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        # before the first CUDA call: the oracle's OpenMP team is created in a clean process
-        import oracle
-        sample = OracleSample(w, min(ORACLE_GROUPS, w.n_groups))
-        sec = min(sample.run() for _ in range(2))
-        cpu_base = {"value": sample.sw.traj_steps / sec, "unit": UNIT, "cores": oracle.num_threads(),
-                    "kind": "oracle", "sample": sample.desc + f"; best of 2 runs, {sec:.1f} s each"}
-        del sample
-
-    torch.cuda.set_device(local)
-    dist = None
-    if world > 1 or "TORCHELASTIC_RUN_ID" in os.environ:      # launched by torch.distributed.run
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    if rank == 0:
-        from paper_2512_15347_b200 import build as pg_build
-        pg_build.build()                 # no-op when libprogrpo.so is up to date; raises if nvcc fails
-    if dist is not None:
-        dist.barrier()
-    B.lib()
-    dev = torch.device("cuda", local)
-    from dataclasses import replace
-    wr = replace(w, seed=w.seed + 1000 * rank)
-
-    dt = torch.bfloat16 if w.vel_dtype == "bf16" else torch.float32
-    ro = Rollout(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, dt, adv_eps=w.adv_eps,
-                 group_offset=sharding.weak_shard(w.n_groups, rank)[0])
     x0 = wl.initial_latents(wr, device=dev)
-    ext = fin = None
+    ext = fin = vels = None
     if w.velocity == "affine":
         a_c, b_c = wl.affine_field(wr, device=dev)
         velocity = lambda s, x: wl.affine_velocity(x, a_c, b_c)   # stand-in network, inside the timing
@@ -243,6 +222,112 @@ def run_ours(args):
             return table[(ids - base).long()]
         ext = lambda stage: lookup(tables[stage])
         fin = lambda: lookup(tables[-1])
+    return x0, velocity, ext, fin, vels
+
+
+def _other_workload(name, dev, reps, peak):
+    """One of the smaller workloads through the same step-by-step driver: ms per rollout,
+    latent-steps/s and the step kernel's algorithmic GB/s (CUDA events around every call)."""
+    import torch
+    from paper_2512_15347_b200 import workloads as wl
+    from paper_2512_15347_b200.rollout import Rollout
+    w = wl.WORKLOADS[name]
+    dt = torch.bfloat16 if w.vel_dtype == "bf16" else torch.float32
+    ro = Rollout(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, dt, adv_eps=w.adv_eps)
+    x0, velocity, ext, fin, vels = _gpu_inputs(w, w, ro, dev, 0)
+    run = lambda trace=None: ro.run(x0, w.step_coef, w.preview_coef, velocity, external_scores=ext,
+                                    final_rewards=fin, trace=trace)
+    for _ in range(3):
+        run()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    traces = []
+    a.record()
+    for _ in range(reps):
+        tr = []
+        run(trace=tr)
+        traces.append(tr)
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / reps
+    step_ms = sum(e0.elapsed_time(e1) for tr in traces for kind, _, e0, e1 in tr if kind == "step") / reps
+    step_gbs = w.traj_steps * (w.elems * (8 + (2 if w.vel_dtype == "bf16" else 4)) + 4) / (step_ms * 1e-3) / 1e9
+    state_mb = w.n_groups * w.n_expand * w.elems * 4 / 1e6
+    graph = None
+    if w.velocity == "normal" and w.scores == "preview":
+        # the whole rollout as one library call, captured once in a CUDA graph and replayed
+        from paper_2512_15347_b200.rollout import NativeRollout
+        nat = NativeRollout(ro, [w.step_coef(s) for s in range(w.n_steps)],
+                            [w.preview_coef(s) for s, _ in w.stages], vels)
+        nat.capture(x0)
+        nat.graph.replay()
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            nat.graph.replay()
+        b.record()
+        torch.cuda.synchronize()
+        gms = a.elapsed_time(b) / reps
+        graph = {"ms_per_rollout": gms, "latent_steps_per_s": w.traj_steps / (gms * 1e-3)}
+        del nat
+    ro.close()
+    return {"ms_per_rollout": ms, "cuda_graph_replay": graph, "latent_steps_per_s": w.traj_steps / (ms * 1e-3), "step_gbs": step_gbs,
+            "step_frac_of_peak": step_gbs / peak,
+            "regime": ("HBM-streaming" if state_mb > 256 else
+                       f"state {state_mb:.1f} MB fits L2: launch-bound, GB/s is L2-assisted")}
+
+
+
+def run_ours(args):
+    import torch
+    from paper_2512_15347_b200 import binding as B
+    from paper_2512_15347_b200 import workloads as wl
+    from paper_2512_15347_b200 import sharding
+    from paper_2512_15347_b200.rollout import Rollout
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    w = wl.WORKLOADS[args.workload]
+    if args.groups:
+        w = wl.scaled(w, n_groups=args.groups, name=f"{w.name}[{args.groups} groups]")
+
+    cpu_base, cpu_others = None, {}
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        # before the first CUDA call: the oracle's OpenMP team is created in a clean process
+        import oracle
+        sample = OracleSample(w, min(ORACLE_GROUPS, w.n_groups))
+        sec = min(sample.run() for _ in range(2))
+        cpu_base = {"value": sample.sw.traj_steps / sec, "unit": UNIT, "cores": oracle.num_threads(),
+                    "kind": "oracle", "sample": sample.desc + f"; best of 2 runs, {sec:.1f} s each"}
+        del sample
+        if args.workload == "large" and not args.groups and not args.no_others:
+            for name, groups in OTHER_WORKLOADS:
+                ow = wl.WORKLOADS[name]
+                sm = OracleSample(ow, min(groups, ow.n_groups))
+                sec = min(sm.run() for _ in range(2))
+                cpu_others[name] = {"value": sm.sw.traj_steps / sec, "sample": sm.desc}
+                del sm
+
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1 or "TORCHELASTIC_RUN_ID" in os.environ:      # launched by torch.distributed.run
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        from paper_2512_15347_b200 import build as pg_build
+        pg_build.build()                 # no-op when libprogrpo.so is up to date; raises if nvcc fails
+    if dist is not None:
+        dist.barrier()
+    B.lib()
+    dev = torch.device("cuda", local)
+    from dataclasses import replace
+    wr = replace(w, seed=w.seed + 1000 * rank)
+
+    dt = torch.bfloat16 if w.vel_dtype == "bf16" else torch.float32
+    ro = Rollout(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, dt, adv_eps=w.adv_eps,
+                 group_offset=sharding.weak_shard(w.n_groups, rank)[0])
+    x0, velocity, ext, fin, vels = _gpu_inputs(w, wr, ro, dev, rank)
     torch.cuda.synchronize()
 
     def one_rollout(trace=None):
@@ -412,6 +497,16 @@ def run_ours(args):
                  "note": "pg_compact gathers the first stage's survivors (fp32 rows); pg_preview writes "
                          "the bf16 look-ahead latent for an external decoder"}
 
+    # the three smaller workloads, same driver (secondary lines; the bench line is the large one)
+    others = None
+    if rank == 0 and world == 1 and args.workload == "large" and not args.groups and not args.no_others:
+        others = {}
+        for name, _ in OTHER_WORKLOADS:
+            others[name] = _other_workload(name, dev, max(5, min(args.steps, 20)), peak)
+            if name in cpu_others:
+                others[name]["cpu_oracle_latent_steps_per_s"] = cpu_others[name]["value"]
+                others[name]["cpu_oracle_sample"] = cpu_others[name]["sample"]
+
     # end to end through the host-buffer entry point (pinned host memory, copies inside the timing)
     e2e = None
     if not args.no_e2e:
@@ -438,7 +533,7 @@ def run_ours(args):
                                 v["launches"] // args.steps} for k, v in kinds.items()},
                 "score_gbs": score_gbs, "prune_stage_gbs": prune_stage_gbs,
                 "hbm_gbs_whole_rollout": (step_bytes + (score_bytes if score_gbs else 0)) / (total_ms * 1e-3) / 1e9,
-                "ovf_microbench": ovf, "drivers": drivers, "policy_update": policy, "other_kernels": other, "e2e": e2e, "cpu_baseline": cpu_base}
+                "ovf_microbench": ovf, "drivers": drivers, "policy_update": policy, "other_kernels": other, "other_workloads": others, "e2e": e2e, "cpu_baseline": cpu_base}
         print(json.dumps(line))
     ro.close()
     if dist is not None:
@@ -531,6 +626,7 @@ def main():
                     help="prompt groups per GPU (default: the workload's own; smaller for profiling)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-others", action="store_true", help="skip the three smaller workloads")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
