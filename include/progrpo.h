@@ -370,6 +370,17 @@ int pg_rollout_run(pg_rollout *h, const pg_step_coef *step_coef, const pg_previe
  * memory) to `dst` (device) in stream order. */
 int pg_rollout_traj_ids(pg_rollout *h, int32_t *dst, void *stream);
 
+/*
+ * Diagnostic (the paper has no counterpart): exercises the library's bounded device-side wait.
+ * The only wait inside the kernels is the selection kernel's wait for its score rows to land in
+ * shared memory; it gives up after a fixed number of attempts, sets status bit 1 and lets the
+ * kernel return, so that a lost copy shows up as PG_ETIMEOUT from pg_rollout_status instead of a
+ * hung GPU.  This call launches one warp that waits the same way on a barrier nothing completes:
+ * the wait runs out (a fraction of a second at most), bit 1 of the handle's status word is set,
+ * and the next pg_rollout_status returns PG_ETIMEOUT.  pg_rollout_reset clears the word.
+ */
+int pg_selftest_bounded_wait(pg_rollout *h, void *stream);
+
 /* Raw Philox4x32-10 blocks for n (counter, key) pairs: ctr [n,4], key [n,2],
  * out [n,4] uint32 device arrays.  Exposes the library's generator so that it
  * can be compared bit for bit with another implementation. */

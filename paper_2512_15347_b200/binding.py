@@ -96,6 +96,7 @@ def lib() -> ctypes.CDLL:
                                  ctypes.POINTER(vp), ctypes.POINTER(vp), vp, vp, sz,
                                  ctypes.POINTER(RolloutOutputs), vp]
     L.pg_rollout_traj_ids.argtypes = [vp, vp, vp]
+    L.pg_selftest_bounded_wait.argtypes = [vp, vp]
     L.pg_philox_raw.argtypes = [i64, vp, vp, vp, vp]
     L.pg_normal_rows.argtypes = [u64, i32, i32, i32, i32, vp, vp, vp]
     L.pg_strerror.argtypes = [ctypes.c_int]
@@ -254,6 +255,11 @@ def score_static(n_rows: int, elems: int, vel_dtype: int, coef, x, vel, scores_o
     c = PreviewCoef(*coef)
     _check(lib().pg_score_static(n_rows, elems, vel_dtype, ctypes.byref(c), _p(x), _p(vel),
                                  _p(scores_out), _stream(stream)), "pg_score_static")
+
+
+def selftest_bounded_wait(h: int, stream=None) -> None:
+    """Makes the library's bounded device-side wait run out once (sets status bit 1)."""
+    _check(lib().pg_selftest_bounded_wait(h, _stream(stream)), "pg_selftest_bounded_wait")
 
 
 def rollout_traj_ids(h: int, dst, stream=None) -> None:

@@ -103,6 +103,25 @@ __device__ __forceinline__ float normal_pair(uint32_t r0, uint32_t r1, float& a,
   return neg2ln;
 }
 
+// Bounded wait on an mbarrier in shared memory (`bar` = shared-space address) for the phase of
+// the given parity: up to `limit` try_wait attempts.  Returns true once the phase has completed,
+// false when the attempts ran out - the caller then records the timeout and leaves; no wait in
+// this library is unbounded.
+__device__ __forceinline__ bool mbarrier_wait_bounded(unsigned int bar, unsigned int parity, int limit) {
+  unsigned int done = 0;
+  for (int it = 0; it < limit && !done; ++it) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+  }
+  return done != 0;
+}
+constexpr int kBulkWaitLimit = 1 << 14;   // try_wait attempts per round before giving up
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
@@ -285,6 +304,8 @@ int launch_compact(int n_groups, int n_prev, int k, const int32_t* keep_idx, con
                    void* dst, size_t row_bytes, cudaStream_t stream, int32_t* status = nullptr);
 
 int launch_iota(int32_t* dst, int n, int32_t base, cudaStream_t stream);
+
+int launch_wait_selftest(int32_t* status, cudaStream_t stream);
 
 int launch_philox_raw(int64_t n, const uint32_t* ctr, const uint32_t* key, uint32_t* out,
                       cudaStream_t stream);

@@ -67,7 +67,6 @@ __device__ __forceinline__ double arithmetic_value(float s) {
 //     the single division are spread over the lanes.
 // warps (= groups) per CTA: four while the per-warp shared memory allows it, one for wide groups
 template <int E> struct OvfWarps { static constexpr int value = (E <= 8) ? 4 : 1; };
-constexpr int kBulkWaitLimit = 1 << 14;   // mbarrier try_wait attempts before giving up
 
 __device__ __forceinline__ float key_to_score(uint32_t key) {
   const uint32_t b = (key & 0x80000000u) ? (key ^ 0x80000000u) : ~key;
@@ -111,17 +110,9 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
           "l"(src), "r"(stage_bytes), "r"(bar)
           : "memory");
     }
-    unsigned int done = 0;
+    bool done = false;
     for (int round = 0; round < 2 && !done; ++round) {
-      for (int it = 0; it < kBulkWaitLimit && !done; ++it) {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done)
-            : "r"(bar), "r"(0u)
-            : "memory");
-      }
+      done = mbarrier_wait_bounded(bar, 0u, kBulkWaitLimit);
       if (!done && round == 0 && threadIdx.x == 0 && p.status) atomicOr(p.status, 2);
     }
     if (!done) return;        // waited twice without success: leave, the host reads the status
@@ -498,6 +489,33 @@ int launch_uniform_select(int n_groups, int n, int k, uint64_t seed, uint32_t st
   uniform_select_kernel<<<n_groups, kOvfThreads, 0, stream>>>(make_philox_keys(seed), n, k, stage,
                                                               group_offset, keep_idx, src_rows, traj_in,
                                                               traj_out);
+  PG_LAUNCH_CHECK();
+  return PG_OK;
+}
+
+// ---------------------------------------------------------------- bounded-wait self-test
+
+// One CTA waits, exactly as the selection kernel waits for its staged rows, on an mbarrier whose
+// phase nothing will ever complete (no copy is issued, nobody arrives).  Both rounds of attempts
+// run out, status bit 1 is set after the first, and the kernel returns normally: the path a lost
+// copy would take, exercised without losing one.
+__global__ void __launch_bounds__(32) wait_selftest_kernel(int32_t* status) {
+  __shared__ __align__(8) unsigned long long bar_mem;
+  const unsigned int bar = (unsigned int)__cvta_generic_to_shared(&bar_mem);
+  if (threadIdx.x == 0) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  bool done = false;
+  for (int round = 0; round < 2 && !done; ++round) {
+    done = mbarrier_wait_bounded(bar, 0u, kBulkWaitLimit);
+    if (!done && round == 0 && threadIdx.x == 0 && status) atomicOr(status, 2);
+  }
+}
+
+int launch_wait_selftest(int32_t* status, cudaStream_t stream) {
+  wait_selftest_kernel<<<1, 32, 0, stream>>>(status);
   PG_LAUNCH_CHECK();
   return PG_OK;
 }

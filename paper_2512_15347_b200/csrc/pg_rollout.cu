@@ -338,6 +338,11 @@ int pg_rollout_traj_ids(pg_rollout* h, int32_t* dst, void* stream) {
   return PG_OK;
 }
 
+int pg_selftest_bounded_wait(pg_rollout* h, void* stream) {
+  if (!h) return PG_EINVAL;
+  return pg::launch_wait_selftest(h->d_status, (cudaStream_t)stream);
+}
+
 int pg_philox_raw(int64_t n, const uint32_t* ctr, const uint32_t* key, uint32_t* out, void* stream) {
   if (n < 0 || (n > 0 && (!ctr || !key || !out)) || !aligned16(out)) return PG_EINVAL;
   return pg::launch_philox_raw(n, ctr, key, out, (cudaStream_t)stream);

@@ -514,6 +514,29 @@ def test_empty_batches_are_accepted(B):
     torch.cuda.synchronize()
 
 
+def test_bounded_wait_runs_out_and_is_reported(B):
+    """The device-side wait gives up instead of hanging: a wait that nothing completes ends by
+    itself, the status word reports it, and the handle stays usable afterwards."""
+    G, N0, d = 2, 8, 64
+    h, _ = _handle(B, G, N0, d, T=2, stages=[(0, 4)])
+    try:
+        assert B.rollout_status(h) == (G * N0, 0, 0)
+        B.selftest_bounded_wait(h)
+        with pytest.raises(B.PgError) as e:
+            B.rollout_status(h)
+        assert e.value.code == B.ETIMEOUT
+        assert B.rollout_status(h, raise_on_flags=False)[2] == 2
+        B.rollout_reset(h)
+        sc = np.arange(G * N0, dtype=np.float32).reshape(G, N0)
+        keep = torch.empty(G * 4, dtype=torch.int32, device="cuda")
+        B.prune_ovf(h, 0, U.to_dev(sc), keep)
+        assert B.rollout_status(h) == (G * 4, 0, 0)
+        np.testing.assert_array_equal(keep.cpu().numpy().reshape(G, 4), oracle.ovf_select(sc, 4)[0])
+    finally:
+        torch.cuda.synchronize()
+        B.rollout_destroy(h)
+
+
 # ------------------------------------------------------------------ diagnostics and the uniform baseline
 
 def test_group_stats_match_oracle(B):
