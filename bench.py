@@ -270,6 +270,22 @@ def _other_workload(name, dev, reps, peak):
         gms = a.elapsed_time(b) / reps
         graph = {"ms_per_rollout": gms, "latent_steps_per_s": w.traj_steps / (gms * 1e-3)}
         del nat
+    elif w.velocity == "affine" and w.scores == "preview":
+        # predictions depend on the latents: the step-by-step driver with the stand-in network's
+        # torch ops recorded into one CUDA graph
+        from paper_2512_15347_b200.rollout import GraphedRollout
+        gr = GraphedRollout(ro, x0, w.step_coef, w.preview_coef, velocity)
+        gr.replay()
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(reps):
+            gr.replay()
+        b.record()
+        torch.cuda.synchronize()
+        gms = a.elapsed_time(b) / reps
+        graph = {"ms_per_rollout": gms, "latent_steps_per_s": w.traj_steps / (gms * 1e-3),
+                 "note": "stand-in network (2 torch ops per step) inside the graph"}
+        del gr
     ro.close()
     return {"ms_per_rollout": ms, "cuda_graph_replay": graph, "latent_steps_per_s": w.traj_steps / (ms * 1e-3), "step_gbs": step_gbs,
             "step_frac_of_peak": step_gbs / peak,

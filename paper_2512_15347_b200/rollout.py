@@ -247,3 +247,33 @@ class NativeRollout:
         if ws_lo <= o.rewards < ws_hi:
             out.rewards = self._view(o.rewards, n, torch.float32)
         return out
+
+
+class GraphedRollout:
+    """The step-by-step driver recorded once into a CUDA graph and replayed, network included.
+
+    For launch-bound rollouts whose predictions depend on the current latents (a denoiser, or a
+    stand-in such as an affine field, written as capturable torch ops): ``velocity(step, x)`` and
+    the optional score / reward callbacks are traced during capture, so a replay re-runs the
+    library's kernels and the network's kernels from x0's current contents without any Python in
+    between.  The callbacks must not synchronise or move data to the host."""
+
+    def __init__(self, ro: Rollout, x0: torch.Tensor, step_coef, preview_coef, velocity,
+                 external_scores=None, final_rewards=None):
+        self.ro, self.x0 = ro, x0
+        run = lambda: ro.run(x0, step_coef, preview_coef, velocity, external_scores=external_scores,
+                             final_rewards=final_rewards)
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(side):
+            run()                                   # warm-up outside the capture (loads kernels)
+        torch.cuda.current_stream().wait_stream(side)
+        torch.cuda.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            self.out = run()
+
+    def replay(self) -> RolloutOutput:
+        self.graph.replay()
+        return self.out
+

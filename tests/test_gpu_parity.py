@@ -738,6 +738,34 @@ def test_out_of_range_gather_indices_are_reported_not_dereferenced(B):
         B.rollout_destroy(h)
 
 
+def test_graphed_stepwise_rollout_with_a_network_in_the_loop(B):
+    """The tiny workload (predictions computed from the current latents by torch ops) captured
+    into a CUDA graph: replays reproduce the step-by-step run bit for bit, also after x0 changes."""
+    from paper_2512_15347_b200.rollout import GraphedRollout
+    w = wl.WORKLOADS["tiny"]
+    inp = U.SharedInputs(w)
+    ro, out = U.run_gpu(w, inp)
+    want = [t.clone() for t in (out.x_final, torch.cat(out.logp), out.stage_keep[0], out.adv, out.traj_id)]
+    a, b = (t.cuda() for t in inp.affine)
+    x0 = U.to_dev(inp.x0)
+    g = GraphedRollout(ro, x0, w.step_coef, w.preview_coef, lambda s, x: wl.affine_velocity(x, a, b))
+
+    def same(o, ref):
+        torch.cuda.synchronize()
+        got = (o.x_final, torch.cat(o.logp), o.stage_keep[0], o.adv, o.traj_id)
+        return all(torch.equal(p, q) for p, q in zip(got, ref))
+
+    assert same(g.replay(), want) and same(g.replay(), want)
+    x0.mul_(-1.0)                                      # new initial latents, same graph
+    o = g.replay()
+    torch.cuda.synchronize()
+    assert not torch.equal(o.x_final, want[0])
+    ro2, out2 = U.run_gpu(w, type("I", (), {"x0": -inp.x0, "vel_device": inp.vel_device})())
+    assert same(o, (out2.x_final, torch.cat(out2.logp), out2.stage_keep[0], out2.adv, out2.traj_id))
+    ro2.close()
+    ro.close()
+
+
 def test_initial_latents_from_the_library_generator(B):
     from paper_2512_15347_b200.rollout import initial_latents
     G, N0, d = 3, 5, 4096
