@@ -57,9 +57,9 @@ def test_normals_match_oracle(B):
 # ------------------------------------------------------------------ step
 
 @pytest.mark.parametrize("bf16", [False, True])
-@pytest.mark.parametrize("d", [4, 1000, 8192, 3 * 8192 + 20, 65536])
+@pytest.mark.parametrize("d", [4, 1000, 8192, 3 * 8192 + 20, 65536, 4 * 1024 * 1024 + 8])
 def test_step_matches_oracle(B, bf16, d):
-    n_groups, n0 = 3, 5
+    n_groups, n0 = (3, 5) if d < 1 << 20 else (1, 2)      # the 16 MB latents: two rows, 513 chunks each, the last one ragged
     n = n_groups * n0
     rng = np.random.default_rng(d + bf16)
     x = rng.standard_normal((n, d)).astype(np.float32)
@@ -92,6 +92,30 @@ def test_step_matches_oracle(B, bf16, d):
         B.rollout_destroy(h)
 
 
+def test_step_and_score_with_many_short_rows(B):
+    """70 000 trajectories of 8 elements: one CTA per row, more rows than a 16-bit grid dimension."""
+    G, N0, d = 700, 100, 8
+    n = G * N0
+    rng = np.random.default_rng(11)
+    x = rng.standard_normal((n, d)).astype(np.float32)
+    v = rng.standard_normal((n, d)).astype(np.float32)
+    h, _ = _handle(B, G, N0, d, seed=4)
+    try:
+        x_out = torch.empty(n, d, device="cuda")
+        lp = torch.empty(n, device="cuda")
+        sc = torch.empty(n, device="cuda")
+        x_dev, v_dev = U.to_dev(x), U.to_dev(v)
+        B.score(h, (1.0, 0.5), x_dev, v_dev, sc)
+        B.step(h, 0, (1.0, 0.1, 0.2), x_dev, v_dev, None, x_out, lp)
+        ref_x, ref_lp = oracle.step(x, v, np.arange(n, dtype=np.int32), 4, 0, 1.0, 0.1, 0.2)
+        assert U.latent_err(x_out.cpu().numpy(), ref_x) <= U.LATENT_TOL
+        assert U.logp_err(lp.cpu().numpy(), ref_lp, d) <= U.LOGP_TOL
+        assert np.abs(sc.cpu().numpy() - oracle.score(x, v, 1.0, 0.5)[0]).max() <= 1e-6
+    finally:
+        torch.cuda.synchronize()
+        B.rollout_destroy(h)
+
+
 def test_step_is_reproducible_and_mean_mode(B):
     n, d = 6, 5 * 8192
     x = torch.randn(n, d, device="cuda")
@@ -112,9 +136,9 @@ def test_step_is_reproducible_and_mean_mode(B):
 # ------------------------------------------------------------------ score
 
 @pytest.mark.parametrize("bf16", [False, True])
-@pytest.mark.parametrize("d", [4, 1000, 8192, 3 * 8192 + 20, 262144])
+@pytest.mark.parametrize("d", [4, 1000, 8192, 3 * 8192 + 20, 262144, 4 * 1024 * 1024 + 8])
 def test_score_matches_oracle(B, bf16, d):
-    n_groups, n0 = 2, 4
+    n_groups, n0 = (2, 4) if d < 1 << 20 else (1, 2)
     n = n_groups * n0
     rng = np.random.default_rng(d + 10 * bf16)
     x = rng.standard_normal((n, d)).astype(np.float32) + 0.3
