@@ -358,6 +358,43 @@ def test_scaled_rollout_matches_oracle(B, name, groups, elems):
     ro.close()
 
 
+def test_group_shards_reproduce_the_unsharded_rollout(B):
+    """Multi-GPU layout on one device: the groups dealt out to two ranks (3 + 2), each shard run
+    with its own handle and global group offset, give the unsharded rollout bit for bit - latents,
+    log-probs, kept slots, advantages, trajectory ids."""
+    from paper_2512_15347_b200 import sharding
+    from paper_2512_15347_b200.rollout import Rollout
+    total = 5
+    w = wl.scaled(wl.WORKLOADS["large"], n_groups=total, elems=8192 + 512)
+    inp = U.SharedInputs(w)
+    ro, whole = U.run_gpu(w, inp)
+    x0 = U.to_dev(inp.x0)
+    parts = []
+    for rank in range(2):
+        first, count = sharding.group_shard(total, 2, rank)
+        sh = Rollout(count, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, torch.bfloat16,
+                     adv_eps=w.adv_eps, group_offset=first)
+
+        def vel(s, x, first=first, count=count):
+            per = w.rows_before(s)
+            full = U.vel_to_dev(inp.vel_numpy(s, np.empty((total * per, 0))))
+            return full[first * per:(first + count) * per].contiguous()
+
+        o = sh.run(x0[first * w.n_expand:(first + count) * w.n_expand], w.step_coef, w.preview_coef, vel)
+        torch.cuda.synchronize()
+        parts.append((o.x_final.clone(), [t.clone() for t in o.logp], [t.clone() for t in o.stage_keep],
+                      o.adv.clone(), o.traj_id.clone()))
+        sh.close()
+    assert torch.equal(torch.cat([p[0] for p in parts]), whole.x_final)
+    for s in range(w.n_steps):
+        assert torch.equal(torch.cat([p[1][s] for p in parts]), whole.logp[s])
+    for i in range(len(w.stages)):
+        assert torch.equal(torch.cat([p[2][i] for p in parts]), whole.stage_keep[i])
+    assert torch.equal(torch.cat([p[3] for p in parts]), whole.adv)
+    assert torch.equal(torch.cat([p[4] for p in parts]), whole.traj_id)
+    ro.close()
+
+
 def test_resume_from_saved_state(B):
     """Noise is keyed by (seed, trajectory, step, element): restarting from a saved latent at
     step s reproduces the uninterrupted run bit for bit."""
