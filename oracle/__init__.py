@@ -301,6 +301,37 @@ def rollout(x0: np.ndarray, n_groups: int, n_expand: int, n_steps: int,
     return res
 
 
+def survivor_rows(n_groups: int, n_expand: int, n_steps: int, stages: Sequence[Tuple[int, int]],
+                  stage_keep: Sequence[np.ndarray]) -> np.ndarray:
+    """Where the final survivors sat at every step (Section 5.1; Eq. pro_grpo_method sums over the
+    survivors only, but over all T steps, so their log-probs and latents from before a prune must
+    be found among the rows that were active then).
+
+    Written as the definition: every group carries the list of original slots of its active rows
+    through the schedule (a prune at step s replaces the list by its kept entries, in ascending
+    slot order, before step s is taken); afterwards every final survivor is looked up by identity
+    in each step's list.  stage_keep[i] is the [G, k_i] slot list of stage i.  Returns int32
+    [T, G*K]: rows[t][g*K + j] = row (group-major among the rows active at step t) of the j-th
+    final survivor of group g.
+    """
+    stage_at = {int(s): i for i, (s, _) in enumerate(stages)}
+    active = [list(range(n_expand)) for _ in range(n_groups)]
+    per_step = []
+    for t in range(n_steps):
+        if t in stage_at:
+            keep = np.asarray(stage_keep[stage_at[t]]).reshape(n_groups, -1)
+            active = [[active[g][int(i)] for i in keep[g]] for g in range(n_groups)]
+        per_step.append([list(a) for a in active])
+    k_final = len(active[0])
+    rows = np.empty((n_steps, n_groups * k_final), dtype=np.int32)
+    for t in range(n_steps):
+        k_t = len(per_step[t][0])
+        for g in range(n_groups):
+            for j, orig in enumerate(active[g]):
+                rows[t, g * k_final + j] = g * k_t + per_step[t][g].index(orig)
+    return rows
+
+
 # ---------------------------------------------------------------- policy update (Eq. ratio_method, Eq. pro_grpo_method)
 
 def policy_logprob(x: np.ndarray, x_next: np.ndarray, vel: np.ndarray, vel_ref: Optional[np.ndarray],
