@@ -61,6 +61,7 @@ extern "C" {
 #define PG_VEL_BF16 1
 
 #define PG_MAX_GROUP 1024   /* largest N0 (trajectories per group) the selection kernels take */
+#define PG_MAX_STAGES 32    /* most pruning checkpoints pg_survivor_rows can trace back through */
 
 typedef struct pg_rollout pg_rollout; /* opaque */
 
@@ -369,6 +370,32 @@ int pg_rollout_run(pg_rollout *h, const pg_step_coef *step_coef, const pg_previe
 /* Copies the handle's current trajectory-id map ([n_active] int32, device
  * memory) to `dst` (device) in stream order. */
 int pg_rollout_traj_ids(pg_rollout *h, int32_t *dst, void *stream);
+
+/*
+ * The survivors' history (Section 5.1, "GRPO with the pruned trajectory set"): the objective of
+ * Eq. "pro_grpo_method" runs over the final survivors only, but over all T steps, so a trainer
+ * needs the survivors' log-probs and latents also from the steps before a prune, when they sat
+ * among rows that were dropped later.
+ *
+ * pg_survivor_rows: rows_out [T, G*K] int32 (device); rows_out[t][g*K + j] is the row, among the
+ *   G*K_t rows that took step t (group-major), of the j-th final survivor of group g.  Depends
+ *   only on the handle's schedule and on keep_idx_packed: the kept-slot lists of all stages as
+ *   pg_prune_ovf wrote them, packed stage after stage ([G*k_1], [G*k_2], ...; device; may be NULL
+ *   without stages), not on the cursor.  A kept slot outside its group is not followed: status
+ *   bit 2 / PG_EINDEX.  More than PG_MAX_STAGES stages: PG_ECAPACITY.
+ * pg_survivor_logp: logp_out [T, G*K] fp32 = the survivors' entries of the per-step log-prob
+ *   arrays packed step after step (logp_packed, sum over t of G*K_t entries, as pg_rollout_run
+ *   and pg_rollout_host lay them out), picked through `rows` from pg_survivor_rows.
+ * pg_gather_rows: dst row j = src row rows[j] for j < n_out (rows of row_bytes bytes, src has
+ *   n_in rows, no overlap): with rows_out[t-1] (or the survivors' original rows for t = 0) this
+ *   collects the survivors' x_t from a stored step.  Out-of-range entries are skipped and
+ *   reported as PG_EINDEX by pg_rollout_status.
+ */
+int pg_survivor_rows(pg_rollout *h, const int32_t *keep_idx_packed, int32_t *rows_out, void *stream);
+int pg_survivor_logp(pg_rollout *h, const int32_t *rows, const float *logp_packed, float *logp_out,
+                     void *stream);
+int pg_gather_rows(pg_rollout *h, const int32_t *rows, int32_t n_out, int32_t n_in, const void *src,
+                   void *dst, size_t row_bytes, void *stream);
 
 /*
  * Diagnostic (the paper has no counterpart): exercises the library's bounded device-side wait.

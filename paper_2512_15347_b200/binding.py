@@ -97,6 +97,9 @@ def lib() -> ctypes.CDLL:
                                  ctypes.POINTER(RolloutOutputs), vp]
     L.pg_rollout_traj_ids.argtypes = [vp, vp, vp]
     L.pg_selftest_bounded_wait.argtypes = [vp, vp]
+    L.pg_survivor_rows.argtypes = [vp, vp, vp, vp]
+    L.pg_survivor_logp.argtypes = [vp, vp, vp, vp, vp]
+    L.pg_gather_rows.argtypes = [vp, vp, i32, i32, vp, vp, sz, vp]
     L.pg_philox_raw.argtypes = [i64, vp, vp, vp, vp]
     L.pg_normal_rows.argtypes = [u64, i32, i32, i32, i32, vp, vp, vp]
     L.pg_strerror.argtypes = [ctypes.c_int]
@@ -255,6 +258,22 @@ def score_static(n_rows: int, elems: int, vel_dtype: int, coef, x, vel, scores_o
     c = PreviewCoef(*coef)
     _check(lib().pg_score_static(n_rows, elems, vel_dtype, ctypes.byref(c), _p(x), _p(vel),
                                  _p(scores_out), _stream(stream)), "pg_score_static")
+
+
+def survivor_rows(h: int, keep_idx_packed, rows_out, stream=None) -> None:
+    """rows_out [T, G*K] int32: row of every final survivor at every step."""
+    _check(lib().pg_survivor_rows(h, _p(keep_idx_packed), _p(rows_out), _stream(stream)), "pg_survivor_rows")
+
+
+def survivor_logp(h: int, rows, logp_packed, logp_out, stream=None) -> None:
+    """logp_out [T, G*K]: the survivors' entries of the packed per-step log-probs."""
+    _check(lib().pg_survivor_logp(h, _p(rows), _p(logp_packed), _p(logp_out), _stream(stream)),
+           "pg_survivor_logp")
+
+
+def gather_rows(h: int, rows, n_out: int, n_in: int, src, dst, row_bytes: int, stream=None) -> None:
+    _check(lib().pg_gather_rows(h, _p(rows), n_out, n_in, _p(src), _p(dst), row_bytes, _stream(stream)),
+           "pg_gather_rows")
 
 
 def selftest_bounded_wait(h: int, stream=None) -> None:

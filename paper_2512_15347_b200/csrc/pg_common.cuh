@@ -303,6 +303,14 @@ int launch_advantages(int n_groups, int K, const float* rewards, float eps, floa
 int launch_compact(int n_groups, int n_prev, int k, const int32_t* keep_idx, const void* src,
                    void* dst, size_t row_bytes, cudaStream_t stream, int32_t* status = nullptr);
 
+int launch_survivor_rows(int n_groups, int n_expand, int n_steps, int n_stages, const int32_t* stage_step,
+                         const int32_t* stage_keep, const int32_t* keep_idx, int32_t* rows_out,
+                         int32_t* status, cudaStream_t stream);
+
+int launch_survivor_logp(const int32_t* rows, const float* logp_packed, float* logp_out,
+                         const long long* step_off_dev, int n_steps, int n_final, int32_t* status,
+                         cudaStream_t stream);
+
 int launch_iota(int32_t* dst, int n, int32_t base, cudaStream_t stream);
 
 int launch_wait_selftest(int32_t* status, cudaStream_t stream);

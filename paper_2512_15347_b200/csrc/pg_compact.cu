@@ -91,4 +91,100 @@ int launch_compact(int n_groups, int n_prev, int k, const int32_t* keep_idx, con
   return PG_OK;
 }
 
+// ---------------------------------------------------------------- survivors' history
+
+// Row of every final survivor at every step.  One thread per final survivor walks the stages
+// from the last to the first: behind stage i its slot is `slot`, in front of it the slot is
+// keep_idx_i[g * k_i + slot].  Steps from stage_step[i] on (up to the next stage) use the slot
+// behind stage i; steps before the first stage use the original slot.
+struct SurvivorParams {
+  const int32_t* keep_idx;      // packed stage after stage: [G * k_0], [G * k_1], ...
+  int32_t* rows_out;            // [T, G * K]
+  int32_t* status;              // bit 2: a kept slot outside its group
+  int n_groups, n_expand, n_steps, n_stages, k_final;
+  int stage_step[PG_MAX_STAGES];
+  int stage_keep[PG_MAX_STAGES];
+  long long stage_off[PG_MAX_STAGES];   // offset of stage i in keep_idx
+};
+
+__global__ void __launch_bounds__(256) survivor_rows_kernel(const __grid_constant__ SurvivorParams p) {
+  const int j = blockIdx.x * blockDim.x + threadIdx.x;
+  const int n_final = p.n_groups * p.k_final;
+  if (j >= n_final) return;
+  const int g = j / p.k_final;
+  int slot = j - g * p.k_final;
+  int t_hi = p.n_steps;                                   // steps [t_lo, t_hi) use the current slot
+  for (int i = p.n_stages - 1; i >= -1; --i) {
+    const int t_lo = i >= 0 ? p.stage_step[i] : 0;
+    const int k_here = i >= 0 ? p.stage_keep[i] : p.n_expand;
+    for (int t = t_lo; t < t_hi; ++t) p.rows_out[(size_t)t * n_final + j] = g * k_here + slot;
+    if (i < 0) break;
+    const int k_before = i > 0 ? p.stage_keep[i - 1] : p.n_expand;
+    const int prev = p.keep_idx[p.stage_off[i] + (long long)g * k_here + slot];
+    if ((unsigned int)prev >= (unsigned int)k_before) {   // never used as an index
+      if (p.status) atomicOr(p.status, 4);
+      slot = 0;
+    } else {
+      slot = prev;
+    }
+    t_hi = t_lo;
+  }
+}
+
+int launch_survivor_rows(int n_groups, int n_expand, int n_steps, int n_stages, const int32_t* stage_step,
+                         const int32_t* stage_keep, const int32_t* keep_idx, int32_t* rows_out,
+                         int32_t* status, cudaStream_t stream) {
+  if (n_stages > PG_MAX_STAGES) return PG_ECAPACITY;
+  SurvivorParams p;
+  p.keep_idx = keep_idx;
+  p.rows_out = rows_out;
+  p.status = status;
+  p.n_groups = n_groups;
+  p.n_expand = n_expand;
+  p.n_steps = n_steps;
+  p.n_stages = n_stages;
+  long long off = 0;
+  for (int i = 0; i < n_stages; ++i) {
+    p.stage_step[i] = stage_step[i];
+    p.stage_keep[i] = stage_keep[i];
+    p.stage_off[i] = off;
+    off += (long long)n_groups * stage_keep[i];
+  }
+  p.k_final = n_stages > 0 ? stage_keep[n_stages - 1] : n_expand;
+  const long long n_final = (long long)n_groups * p.k_final;
+  if (n_final == 0 || n_steps == 0) return PG_OK;
+  survivor_rows_kernel<<<(unsigned)((n_final + 255) / 256), 256, 0, stream>>>(p);
+  PG_LAUNCH_CHECK();
+  return PG_OK;
+}
+
+// logp_out[t][j] = logp_packed[offset of step t + rows[t][j]]: the survivors' log-prob history
+// out of the per-step arrays packed step after step.
+__global__ void __launch_bounds__(256)
+survivor_logp_kernel(const int32_t* __restrict__ rows, const float* __restrict__ logp_packed,
+                     float* __restrict__ logp_out, const long long* __restrict__ step_off,
+                     int n_steps, int n_final, int32_t* status) {
+  const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= (long long)n_steps * n_final) return;
+  const int t = (int)(i / n_final);
+  const long long lo = step_off[t], hi = step_off[t + 1];
+  const long long r = rows[i];
+  if (r < 0 || lo + r >= hi) {
+    if (status) atomicOr(status, 4);
+    return;
+  }
+  logp_out[i] = logp_packed[lo + r];
+}
+
+int launch_survivor_logp(const int32_t* rows, const float* logp_packed, float* logp_out,
+                         const long long* step_off_dev, int n_steps, int n_final, int32_t* status,
+                         cudaStream_t stream) {
+  const long long total = (long long)n_steps * n_final;
+  if (total == 0) return PG_OK;
+  survivor_logp_kernel<<<(unsigned)((total + 255) / 256), 256, 0, stream>>>(rows, logp_packed, logp_out,
+                                                                           step_off_dev, n_steps, n_final, status);
+  PG_LAUNCH_CHECK();
+  return PG_OK;
+}
+
 }  // namespace pg

@@ -37,6 +37,8 @@ struct pg_rollout {
   float* d_partials = nullptr;
   unsigned int* d_tickets = nullptr;
   int32_t* d_status = nullptr;
+  long long* d_step_off = nullptr;   // [T + 1] offsets of the steps in a packed per-step row array
+  long long total_step_rows = 0;
 };
 
 using pg::cuda_fail;
@@ -93,6 +95,18 @@ int pg_rollout_init(const pg_config* cfg, pg_rollout** out) {
   if (e == cudaSuccess) e = cudaMalloc(&h->d_partials, 2 * slots * sizeof(float))   /* up to two sums per row */;
   if (e == cudaSuccess) e = cudaMalloc(&h->d_tickets, rows * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMalloc(&h->d_status, sizeof(int32_t));
+  std::vector<long long> step_off((size_t)cfg->n_steps + 1, 0);
+  {
+    int k = cfg->n_expand, si = 0;
+    for (int s = 0; s < cfg->n_steps; ++s) {
+      if (si < cfg->n_stages && cfg->stage_step[si] == s) k = cfg->stage_keep[si++];
+      step_off[s + 1] = step_off[s] + (long long)cfg->n_groups * k;
+    }
+  }
+  h->total_step_rows = step_off.back();
+  if (e == cudaSuccess) e = cudaMalloc(&h->d_step_off, step_off.size() * sizeof(long long));
+  if (e == cudaSuccess)
+    e = cudaMemcpy(h->d_step_off, step_off.data(), step_off.size() * sizeof(long long), cudaMemcpyHostToDevice);
   if (e == cudaSuccess) e = cudaMemset(h->d_tickets, 0, rows * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMemset(h->d_status, 0, sizeof(int32_t));
   int lrc = PG_OK;
@@ -115,6 +129,7 @@ int pg_rollout_destroy(pg_rollout* h) {
   cudaFree(h->d_partials);
   cudaFree(h->d_tickets);
   cudaFree(h->d_status);
+  cudaFree(h->d_step_off);
   delete h;
   return PG_OK;
 }
@@ -336,6 +351,33 @@ int pg_rollout_traj_ids(pg_rollout* h, int32_t* dst, void* stream) {
                           (size_t)h->cfg.n_groups * h->k_cur * sizeof(int32_t),
                           cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
   return PG_OK;
+}
+
+int pg_survivor_rows(pg_rollout* h, const int32_t* keep_idx_packed, int32_t* rows_out, void* stream) {
+  if (!h || !rows_out) return PG_EINVAL;
+  if (h->cfg.n_stages > 0 && !keep_idx_packed) return PG_EINVAL;
+  return pg::launch_survivor_rows(h->cfg.n_groups, h->cfg.n_expand, h->cfg.n_steps, h->cfg.n_stages,
+                                  h->stage_step.data(), h->stage_keep.data(), keep_idx_packed, rows_out,
+                                  h->d_status, (cudaStream_t)stream);
+}
+
+int pg_survivor_logp(pg_rollout* h, const int32_t* rows, const float* logp_packed, float* logp_out,
+                     void* stream) {
+  if (!h || !rows || !logp_packed || !logp_out) return PG_EINVAL;
+  const int k_final = h->cfg.n_stages > 0 ? h->stage_keep.back() : h->cfg.n_expand;
+  return pg::launch_survivor_logp(rows, logp_packed, logp_out, h->d_step_off, h->cfg.n_steps,
+                                  h->cfg.n_groups * k_final, h->d_status, (cudaStream_t)stream);
+}
+
+int pg_gather_rows(pg_rollout* h, const int32_t* rows, int32_t n_out, int32_t n_in, const void* src,
+                   void* dst, size_t row_bytes, void* stream) {
+  if (!h || n_out < 0 || n_in < 0 || row_bytes == 0) return PG_EINVAL;
+  if (n_out == 0) return PG_OK;
+  if (!rows || !src || !dst || n_in == 0) return PG_EINVAL;
+  const uintptr_t s = (uintptr_t)src, d = (uintptr_t)dst;
+  if (s < d + (size_t)n_out * row_bytes && d < s + (size_t)n_in * row_bytes) return PG_EINVAL;   // overlap
+  // one "group" of n_in rows from which n_out are taken: the compaction kernel's gather
+  return pg::launch_compact(1, n_in, n_out, rows, src, dst, row_bytes, (cudaStream_t)stream, h->d_status);
 }
 
 int pg_selftest_bounded_wait(pg_rollout* h, void* stream) {

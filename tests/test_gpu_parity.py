@@ -575,6 +575,79 @@ def test_empty_batches_are_accepted(B):
     torch.cuda.synchronize()
 
 
+def test_survivor_rows_match_oracle_on_random_schedules(B):
+    rng = np.random.default_rng(5)
+    for trial in range(12):
+        G = int(rng.integers(1, 6))
+        N0 = int(rng.integers(1, 40))
+        T = int(rng.integers(1, 12))
+        n_st = int(rng.integers(0, min(T, 4) + 1))
+        steps = sorted(rng.choice(T, size=n_st, replace=False).tolist())
+        stages, keeps, k_prev = [], [], N0
+        for s_ in steps:
+            k = int(rng.integers(1, k_prev + 1))
+            stages.append((int(s_), k))
+            keeps.append(np.stack([np.sort(rng.choice(k_prev, size=k, replace=False)) for _ in range(G)]).astype(np.int32))
+            k_prev = k
+        h, _ = _handle(B, G, N0, 8, T=T, stages=stages)
+        try:
+            packed = np.concatenate([k.reshape(-1) for k in keeps]) if keeps else np.zeros(1, np.int32)
+            rows = torch.full((T, G * k_prev), -1, dtype=torch.int32, device="cuda")
+            B.survivor_rows(h, U.to_dev(packed) if keeps else None, rows)
+            ref = oracle.survivor_rows(G, N0, T, stages, keeps)
+            np.testing.assert_array_equal(rows.cpu().numpy(), ref, err_msg=f"trial {trial}: {stages}")
+            assert B.rollout_status(h)[2] == 0
+        finally:
+            torch.cuda.synchronize()
+            B.rollout_destroy(h)
+
+
+def test_survivors_history_after_a_pruned_rollout(B):
+    """After a rollout with three prunes: the survivors' log-prob history and their latents of an
+    early step, collected through pg_survivor_rows / _logp / pg_gather_rows, against the oracle's."""
+    from paper_2512_15347_b200.rollout import NativeRollout
+    w = wl.scaled(wl.WORKLOADS["large"], n_groups=3, elems=8192 + 256)
+    inp = U.SharedInputs(w)
+    ref = U.run_oracle(w, inp, keep_steps=True)
+    ro, out = U.run_gpu(w, inp)
+    T, n_final = w.n_steps, w.n_groups * w.final_keep
+    keep_packed = torch.cat(out.stage_keep)
+    logp_packed = torch.cat(out.logp)
+    rows = torch.empty(T, n_final, dtype=torch.int32, device="cuda")
+    hist = torch.empty(T, n_final, device="cuda")
+    B.survivor_rows(ro.h, keep_packed, rows)
+    B.survivor_logp(ro.h, rows, logp_packed, hist)
+    own_keep = [a.cpu().numpy().reshape(w.n_groups, -1) for a in out.stage_keep]
+    np.testing.assert_array_equal(rows.cpu().numpy(),
+                                  oracle.survivor_rows(w.n_groups, w.n_expand, T, w.stages, own_keep))
+    # the values below need the device's selections to be the oracle's (they are, bit-reproducibly,
+    # for this seed; a score gap below the score tolerance could legitimately flip one)
+    assert all(np.array_equal(a, b) for a, b in zip(own_keep, ref.stage_keep))
+    ref_rows = oracle.survivor_rows(w.n_groups, w.n_expand, T, w.stages, ref.stage_keep)
+    ref_hist = np.stack([ref.logp[t][ref_rows[t]] for t in range(T)])
+    assert U.logp_err(hist.cpu().numpy(), ref_hist, w.elems) <= U.LOGP_TOL
+    # the survivors' latents entering step 1 (stored in the 64-per-group layout of step 0)
+    x1 = torch.empty(w.n_groups * w.n_expand, w.elems, device="cuda")
+    lp = torch.empty(w.n_groups * w.n_expand, device="cuda")
+    B.rollout_reset(ro.h)
+    B.step(ro.h, 0, w.step_coef(0), U.to_dev(inp.x0), inp.vel_device(0, torch.empty(w.n_groups * w.n_expand, 0)),
+           None, x1, lp)
+    surv = torch.empty(n_final, w.elems, device="cuda")
+    B.gather_rows(ro.h, rows[0], n_final, w.n_groups * w.n_expand, x1, surv, w.elems * 4)
+    assert U.latent_err(surv.cpu().numpy(), ref.x_steps[0][ref_rows[0]]) <= U.LATENT_TOL
+    assert B.rollout_status(ro.h)[2] == 0
+    # an index outside the source is skipped and reported
+    bad = rows[0].clone()
+    bad[3] = w.n_groups * w.n_expand
+    surv.fill_(7.0)
+    B.gather_rows(ro.h, bad, n_final, w.n_groups * w.n_expand, x1, surv, w.elems * 4)
+    with pytest.raises(B.PgError) as e:
+        B.rollout_status(ro.h)
+    assert e.value.code == B.EINDEX
+    assert torch.all(surv[3] == 7.0)
+    ro.close()
+
+
 def test_bounded_wait_runs_out_and_is_reported(B):
     """The device-side wait gives up instead of hanging: a wait that nothing completes ends by
     itself, the status word reports it, and the handle stays usable afterwards."""
