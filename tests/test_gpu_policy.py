@@ -125,3 +125,57 @@ def test_policy_update_after_a_rollout_has_unit_ratio():
     assert (ratio - 1).abs().max().item() < 1e-5
     assert abs(obj.item()) < 1e-6
     ro.close()
+
+
+def test_policy_update_on_the_survivors_of_a_pruned_rollout():
+    """The whole chain after a rollout with two prunes: the survivors' transitions are collected
+    from the stored steps (rows from pg_survivor_rows, latents and predictions through
+    pg_gather_rows), re-evaluated under the same predictions, and give back the survivors' own
+    log-prob history (pg_survivor_logp): ratio 1 at every step, objective = mean advantage = 0."""
+    from paper_2512_15347_b200 import binding as B
+    from paper_2512_15347_b200.rollout import Rollout
+    w = wl.Workload("upd-pruned", 3, 12, ((1, 6), (3, 2)), 5, 8192 + 512, 1, "bf16", 9, "normal", "preview")
+    inp = U.SharedInputs(w)
+    ro = Rollout(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, torch.bfloat16, logp_mean=True)
+    xs, vels = [], []
+
+    def velocity(s, x):
+        v = inp.vel_device(s, x)
+        xs.append(x.clone())                   # x_s in the layout of the rows alive before any prune at s
+        vels.append(v)
+        return v
+
+    out = ro.run(U.to_dev(inp.x0), w.step_coef, w.preview_coef, velocity)
+    xs.append(out.x_final.clone())
+    T, n = w.n_steps, w.n_groups * w.final_keep
+    rows = torch.empty(T, n, dtype=torch.int32, device="cuda")
+    B.survivor_rows(ro.h, torch.cat(out.stage_keep), rows)
+    lp_old = torch.empty(T, n, device="cuda")
+    B.survivor_logp(ro.h, rows, torch.cat(out.logp), lp_old)
+    orig = (out.traj_id - 0).to(torch.int32)   # group_offset 0: the original row of every survivor
+    lp_new = torch.empty(T, n, device="cuda")
+    d = w.elems
+    for t in range(T):
+        rows_in = orig if t == 0 else rows[t - 1]
+        n_in = xs[t].shape[0]
+        x_t = torch.empty(n, d, device="cuda")
+        v_t = torch.empty(n, d, device="cuda", dtype=torch.bfloat16)
+        B.gather_rows(ro.h, rows_in, n, n_in, xs[t], x_t, d * 4)
+        B.gather_rows(ro.h, rows_in, n, n_in, vels[t], v_t, d * 2)
+        if t + 1 < T:
+            x_n = torch.empty(n, d, device="cuda")
+            B.gather_rows(ro.h, rows[t], n, xs[t + 1].shape[0], xs[t + 1], x_n, d * 4)
+        else:
+            x_n = xs[T]
+        B.policy_logprob(ro.h, w.step_coef(t), x_t, x_n, v_t, None, lp_new[t], None)
+    torch.cuda.synchronize()
+    assert B.rollout_status(ro.h)[2] == 0
+    assert (lp_new - lp_old).abs().max().item() < 2e-6
+    ratio = torch.empty(T, n, device="cuda")
+    dlogp = torch.empty(T, n, device="cuda")
+    obj = torch.empty(1, device="cuda")
+    B.policy_objective(ro.h, T, lp_new, lp_old, None, out.adv, 0.2, 0.0, ratio, dlogp, obj)
+    torch.cuda.synchronize()
+    assert (ratio - 1).abs().max().item() < 1e-5
+    assert abs(obj.item()) < 1e-6
+    ro.close()
