@@ -19,6 +19,8 @@
  *    reduction partials, tickets, status word), all released by
  *    pg_rollout_destroy().  pg_config and the coefficient structs are HOST
  *    memory, read during the call only.
+ *  - A handle belongs to the device that was current when pg_rollout_init created it; every
+ *    call on it must be made with that device current (else PG_EDEVICE, nothing is launched).
  *  - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Calls
  *    enqueue work and return; none synchronises, except pg_rollout_status()
  *    and pg_rollout_host().  All calls on one handle must be issued on one
@@ -56,6 +58,7 @@ extern "C" {
 #define PG_ENOMEM     (-6)  /* host or device allocation for the handle failed         */
 #define PG_EINDEX     (-8)  /* reported by pg_rollout_status(): a gather index was out of range */
 #define PG_ECAPACITY  (-7)  /* request larger than a fixed built-in buffer (pg_score_static) */
+#define PG_EDEVICE    (-9)  /* the handle was created on another device than the current one  */
 
 #define PG_VEL_F32  0
 #define PG_VEL_BF16 1

@@ -14,7 +14,7 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libprogrpo.so")
 
-OK, EINVAL, ESTATE, ECUDA, ENONFINITE, ETIMEOUT, ENOMEM, ECAPACITY, EINDEX = 0, -1, -2, -3, -4, -5, -6, -7, -8
+OK, EINVAL, ESTATE, ECUDA, ENONFINITE, ETIMEOUT, ENOMEM, ECAPACITY, EINDEX, EDEVICE = 0, -1, -2, -3, -4, -5, -6, -7, -8, -9
 STATIC_MAX_ROWS, STATIC_MAX_PARTIALS = 8192, 65536
 VEL_F32, VEL_BF16 = 0, 1
 MAX_GROUP = 1024

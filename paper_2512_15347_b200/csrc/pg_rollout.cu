@@ -45,6 +45,14 @@ using pg::cuda_fail;
 
 static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
 
+// A handle's device memory belongs to the device that was current at pg_rollout_init: a call made
+// with another device current would hand that device pointers it cannot reach.
+static int wrong_device(const pg_rollout* h) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return cuda_fail(cudaGetLastError());
+  return dev == h->device ? PG_OK : PG_EDEVICE;
+}
+
 static int validate_config(const pg_config* c) {
   if (!c) return PG_EINVAL;
   if (c->n_groups < 1 || c->n_expand < 1 || c->n_expand > PG_MAX_GROUP) return PG_EINVAL;
@@ -136,6 +144,7 @@ int pg_rollout_destroy(pg_rollout* h) {
 
 int pg_rollout_reset(pg_rollout* h, void* stream) {
   if (!h) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   cudaStream_t st = (cudaStream_t)stream;
   const int rows = h->cfg.n_groups * h->cfg.n_expand;
   h->stage_cur = 0;
@@ -151,6 +160,7 @@ int pg_rollout_reset(pg_rollout* h, void* stream) {
 int pg_rollout_restore(pg_rollout* h, int32_t next_step, int32_t stages_done, const int32_t* traj_ids,
                        void* stream) {
   if (!h || !traj_ids) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (next_step < 0 || next_step > h->cfg.n_steps || stages_done < 0 || stages_done > h->cfg.n_stages)
     return PG_EINVAL;
   // the cursor must be one the schedule can reach: every stage before next_step is done, and the
@@ -179,6 +189,7 @@ int pg_rollout_restore(pg_rollout* h, int32_t next_step, int32_t stages_done, co
 
 int pg_rollout_status(pg_rollout* h, int32_t* n_active, int32_t* next_step, int32_t* device_status) {
   if (!h) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   PG_CUDA(cudaDeviceSynchronize());
   int32_t st = 0;
   PG_CUDA(cudaMemcpy(&st, h->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost));
@@ -194,6 +205,7 @@ int pg_rollout_status(pg_rollout* h, int32_t* n_active, int32_t* next_step, int3
 int pg_step(pg_rollout* h, int32_t step, const pg_step_coef* coef, const float* x_in,
             const void* vel, const int32_t* src_rows, float* x_out, float* logp_out, void* stream) {
   if (!h || !coef || !x_in || !vel || !x_out || !logp_out) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (!aligned16(x_in) || !aligned16(vel) || !aligned16(x_out)) return PG_EINVAL;
   if (src_rows && x_in == x_out) return PG_EINVAL;
   if (!(coef->noise_std >= 0.0) || !std::isfinite(coef->c_x) || !std::isfinite(coef->c_v) ||
@@ -215,6 +227,7 @@ int pg_step(pg_rollout* h, int32_t step, const pg_step_coef* coef, const float* 
 int pg_score(pg_rollout* h, const pg_preview_coef* coef, const float* x, const void* vel,
              float* scores_out, float* preview_out, void* stream) {
   if (!h || !coef || !x || !scores_out) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (!std::isfinite(coef->p_x) || !std::isfinite(coef->p_v)) return PG_EINVAL;
   if (coef->p_v != 0.0 && !vel) return PG_EINVAL;
   if (!aligned16(x) || !aligned16(vel) || !aligned16(preview_out)) return PG_EINVAL;
@@ -227,6 +240,7 @@ int pg_score(pg_rollout* h, const pg_preview_coef* coef, const float* x, const v
 int pg_preview(pg_rollout* h, const pg_preview_coef* coef, const float* x, const void* vel, void* out,
                int32_t out_dtype, void* stream) {
   if (!h || !coef || !x || !vel || !out) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (out_dtype != PG_VEL_F32 && out_dtype != PG_VEL_BF16) return PG_EINVAL;
   if (!std::isfinite(coef->p_x) || !std::isfinite(coef->p_v)) return PG_EINVAL;
   if (!aligned16(x) || !aligned16(vel) || !aligned16(out)) return PG_EINVAL;
@@ -237,6 +251,7 @@ int pg_preview(pg_rollout* h, const pg_preview_coef* coef, const float* x, const
 int pg_prune_ovf(pg_rollout* h, int32_t stage, const float* scores, int32_t* keep_idx,
                  int32_t* src_rows, float* sel_var, void* stream) {
   if (!h || !scores || !keep_idx) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (stage != h->stage_cur || stage >= h->cfg.n_stages) return PG_ESTATE;
   if (h->stage_step[stage] != h->next_step) return PG_ESTATE;
   const int n = h->k_cur, k = h->stage_keep[stage];
@@ -253,6 +268,7 @@ int pg_prune_ovf(pg_rollout* h, int32_t stage, const float* scores, int32_t* kee
 
 int pg_prune_uniform(pg_rollout* h, int32_t stage, int32_t* keep_idx, int32_t* src_rows, void* stream) {
   if (!h || !keep_idx) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (stage != h->stage_cur || stage >= h->cfg.n_stages) return PG_ESTATE;
   if (h->stage_step[stage] != h->next_step) return PG_ESTATE;
   const int n = h->k_cur, k = h->stage_keep[stage];
@@ -280,6 +296,7 @@ int pg_group_stats(int32_t n_groups, int32_t n, const float* scores, float delta
 int pg_compact(pg_rollout* h, const int32_t* keep_idx, const void* src, void* dst, size_t row_bytes,
                void* stream) {
   if (!h || !keep_idx || !src || !dst || row_bytes == 0) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (h->k_prev == 0) return PG_ESTATE;
   const size_t src_bytes = (size_t)h->cfg.n_groups * h->k_prev * row_bytes;
   const size_t dst_bytes = (size_t)h->cfg.n_groups * h->k_cur * row_bytes;
@@ -292,6 +309,7 @@ int pg_compact(pg_rollout* h, const int32_t* keep_idx, const void* src, void* ds
 int pg_advantages(pg_rollout* h, const float* rewards, float* adv, float* mean, float* std,
                   void* stream) {
   if (!h || !rewards || !adv) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   return pg::launch_advantages(h->cfg.n_groups, h->k_cur, rewards, h->cfg.adv_eps, adv, mean, std,
                                (cudaStream_t)stream);
 }
@@ -299,6 +317,7 @@ int pg_advantages(pg_rollout* h, const float* rewards, float* adv, float* mean, 
 int pg_policy_logprob(pg_rollout* h, const pg_step_coef* coef, const float* x, const float* x_next,
                       const void* vel, const void* vel_ref, float* logp_out, float* kl_out, void* stream) {
   if (!h || !coef || !x || !x_next || !vel || !logp_out) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   if ((vel_ref == nullptr) != (kl_out == nullptr)) return PG_EINVAL;
   if (!aligned16(x) || !aligned16(x_next) || !aligned16(vel) || !aligned16(vel_ref)) return PG_EINVAL;
   if (!(coef->noise_std > 0.0) || !std::isfinite(coef->c_x) || !std::isfinite(coef->c_v) ||
@@ -314,6 +333,7 @@ int pg_policy_objective(pg_rollout* h, int32_t n_steps, const float* logp_new, c
                         const float* kl, const float* adv, float clip_eps, float beta, float* ratio,
                         float* dlogp, float* objective, void* stream) {
   if (!h || n_steps < 1 || !logp_new || !logp_old || !adv || !dlogp || !objective) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (!(clip_eps >= 0.f) || !std::isfinite(beta)) return PG_EINVAL;
   return pg::launch_policy_objective(n_steps, h->cfg.n_groups * h->k_cur, logp_new, logp_old, kl, adv,
                                      clip_eps, beta, ratio, dlogp, objective, (cudaStream_t)stream);
@@ -323,6 +343,7 @@ int pg_policy_backward(pg_rollout* h, const pg_step_coef* coef, const float* x, 
                        const void* vel, const void* vel_ref, const float* dlogp, double dkl,
                        void* grad_vel, void* stream) {
   if (!h || !coef || !x || !x_next || !vel || !dlogp || !grad_vel) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (!aligned16(x) || !aligned16(x_next) || !aligned16(vel) || !aligned16(vel_ref) ||
       !aligned16(grad_vel))
     return PG_EINVAL;
@@ -347,6 +368,7 @@ int pg_ovf_select_batched(int32_t n_groups, int32_t n, int32_t k, const float* s
 
 int pg_rollout_traj_ids(pg_rollout* h, int32_t* dst, void* stream) {
   if (!h || !dst) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   PG_CUDA(cudaMemcpyAsync(dst, h->d_traj[h->traj_cur],
                           (size_t)h->cfg.n_groups * h->k_cur * sizeof(int32_t),
                           cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
@@ -355,6 +377,7 @@ int pg_rollout_traj_ids(pg_rollout* h, int32_t* dst, void* stream) {
 
 int pg_survivor_rows(pg_rollout* h, const int32_t* keep_idx_packed, int32_t* rows_out, void* stream) {
   if (!h || !rows_out) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (h->cfg.n_stages > 0 && !keep_idx_packed) return PG_EINVAL;
   return pg::launch_survivor_rows(h->cfg.n_groups, h->cfg.n_expand, h->cfg.n_steps, h->cfg.n_stages,
                                   h->stage_step.data(), h->stage_keep.data(), keep_idx_packed, rows_out,
@@ -364,6 +387,7 @@ int pg_survivor_rows(pg_rollout* h, const int32_t* keep_idx_packed, int32_t* row
 int pg_survivor_logp(pg_rollout* h, const int32_t* rows, const float* logp_packed, float* logp_out,
                      void* stream) {
   if (!h || !rows || !logp_packed || !logp_out) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   const int k_final = h->cfg.n_stages > 0 ? h->stage_keep.back() : h->cfg.n_expand;
   return pg::launch_survivor_logp(rows, logp_packed, logp_out, h->d_step_off, h->cfg.n_steps,
                                   h->cfg.n_groups * k_final, h->d_status, (cudaStream_t)stream);
@@ -372,6 +396,7 @@ int pg_survivor_logp(pg_rollout* h, const int32_t* rows, const float* logp_packe
 int pg_gather_rows(pg_rollout* h, const int32_t* rows, int32_t n_out, int32_t n_in, const void* src,
                    void* dst, size_t row_bytes, void* stream) {
   if (!h || n_out < 0 || n_in < 0 || row_bytes == 0) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (n_out == 0) return PG_OK;
   if (!rows || !src || !dst || n_in == 0) return PG_EINVAL;
   const uintptr_t s = (uintptr_t)src, d = (uintptr_t)dst;
@@ -382,6 +407,7 @@ int pg_gather_rows(pg_rollout* h, const int32_t* rows, int32_t n_out, int32_t n_
 
 int pg_selftest_bounded_wait(pg_rollout* h, void* stream) {
   if (!h) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   return pg::launch_wait_selftest(h->d_status, (cudaStream_t)stream);
 }
 
@@ -408,6 +434,7 @@ const char* pg_strerror(int code) {
     case PG_ENOMEM: return "out of memory";
     case PG_EINDEX: return "a gather index (src_rows / keep_idx) was out of range; the rows were not read";
     case PG_ECAPACITY: return "request exceeds the capacity of a fixed built-in buffer";
+    case PG_EDEVICE: return "the handle belongs to another device than the current one";
     default: return "unknown error code";
   }
 }
@@ -626,6 +653,7 @@ int pg_rollout_run(pg_rollout* h, const pg_step_coef* step_coef, const pg_previe
   if (!h || !step_coef || !x0 || !vel_steps || !workspace || !out || !aligned16(workspace) ||
       !aligned16(x0))
     return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
   const pg_config* cfg = &h->cfg;
   const RunPlan pl = make_run_plan(cfg);
   if (workspace_bytes < pl.total) return PG_EINVAL;

@@ -34,7 +34,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_error_strings(lib):
-    for code in (0, -1, -2, -3, -4, -5, -6, -7, -8):
+    for code in (0, -1, -2, -3, -4, -5, -6, -7, -8, -9):
         assert B.strerror(code) and "unknown" not in B.strerror(code)
     assert "unknown" in B.strerror(-99)
 
