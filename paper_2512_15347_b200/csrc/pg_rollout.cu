@@ -3,6 +3,8 @@
 // pg_compact.cu; this file only validates, keeps the cursor and enqueues.
 #include "pg_common.cuh"
 
+#include <nvtx3/nvToolsExt.h>
+
 #include <atomic>
 #include <cmath>
 #include <cstdlib>
@@ -44,6 +46,15 @@ struct pg_rollout {
 using pg::cuda_fail;
 
 static bool aligned16(const void* p) { return ((uintptr_t)p & 15) == 0; }
+
+// Named range around a library call for timeline tools (NVTX; a no-op costing a pointer test when
+// no tool is attached).
+struct TraceRange {
+  explicit TraceRange(const char* name) { nvtxRangePushA(name); }
+  ~TraceRange() { nvtxRangePop(); }
+  TraceRange(const TraceRange&) = delete;
+  TraceRange& operator=(const TraceRange&) = delete;
+};
 
 // A handle's device memory belongs to the device that was current at pg_rollout_init: a call made
 // with another device current would hand that device pointers it cannot reach.
@@ -204,6 +215,7 @@ int pg_rollout_status(pg_rollout* h, int32_t* n_active, int32_t* next_step, int3
 
 int pg_step(pg_rollout* h, int32_t step, const pg_step_coef* coef, const float* x_in,
             const void* vel, const int32_t* src_rows, float* x_out, float* logp_out, void* stream) {
+  TraceRange trace_range("pg_step");
   if (!h || !coef || !x_in || !vel || !x_out || !logp_out) return PG_EINVAL;
   if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (!aligned16(x_in) || !aligned16(vel) || !aligned16(x_out)) return PG_EINVAL;
@@ -226,6 +238,7 @@ int pg_step(pg_rollout* h, int32_t step, const pg_step_coef* coef, const float* 
 
 int pg_score(pg_rollout* h, const pg_preview_coef* coef, const float* x, const void* vel,
              float* scores_out, float* preview_out, void* stream) {
+  TraceRange trace_range("pg_score");
   if (!h || !coef || !x || !scores_out) return PG_EINVAL;
   if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (!std::isfinite(coef->p_x) || !std::isfinite(coef->p_v)) return PG_EINVAL;
@@ -239,6 +252,7 @@ int pg_score(pg_rollout* h, const pg_preview_coef* coef, const float* x, const v
 
 int pg_preview(pg_rollout* h, const pg_preview_coef* coef, const float* x, const void* vel, void* out,
                int32_t out_dtype, void* stream) {
+  TraceRange trace_range("pg_preview");
   if (!h || !coef || !x || !vel || !out) return PG_EINVAL;
   if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (out_dtype != PG_VEL_F32 && out_dtype != PG_VEL_BF16) return PG_EINVAL;
@@ -250,6 +264,7 @@ int pg_preview(pg_rollout* h, const pg_preview_coef* coef, const float* x, const
 
 int pg_prune_ovf(pg_rollout* h, int32_t stage, const float* scores, int32_t* keep_idx,
                  int32_t* src_rows, float* sel_var, void* stream) {
+  TraceRange trace_range("pg_prune_ovf");
   if (!h || !scores || !keep_idx) return PG_EINVAL;
   if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (stage != h->stage_cur || stage >= h->cfg.n_stages) return PG_ESTATE;
@@ -267,6 +282,7 @@ int pg_prune_ovf(pg_rollout* h, int32_t stage, const float* scores, int32_t* kee
 }
 
 int pg_prune_uniform(pg_rollout* h, int32_t stage, int32_t* keep_idx, int32_t* src_rows, void* stream) {
+  TraceRange trace_range("pg_prune_uniform");
   if (!h || !keep_idx) return PG_EINVAL;
   if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (stage != h->stage_cur || stage >= h->cfg.n_stages) return PG_ESTATE;
@@ -295,6 +311,7 @@ int pg_group_stats(int32_t n_groups, int32_t n, const float* scores, float delta
 
 int pg_compact(pg_rollout* h, const int32_t* keep_idx, const void* src, void* dst, size_t row_bytes,
                void* stream) {
+  TraceRange trace_range("pg_compact");
   if (!h || !keep_idx || !src || !dst || row_bytes == 0) return PG_EINVAL;
   if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (h->k_prev == 0) return PG_ESTATE;
@@ -308,6 +325,7 @@ int pg_compact(pg_rollout* h, const int32_t* keep_idx, const void* src, void* ds
 
 int pg_advantages(pg_rollout* h, const float* rewards, float* adv, float* mean, float* std,
                   void* stream) {
+  TraceRange trace_range("pg_advantages");
   if (!h || !rewards || !adv) return PG_EINVAL;
   if (const int rc_dev = wrong_device(h)) return rc_dev;
   return pg::launch_advantages(h->cfg.n_groups, h->k_cur, rewards, h->cfg.adv_eps, adv, mean, std,
@@ -316,6 +334,7 @@ int pg_advantages(pg_rollout* h, const float* rewards, float* adv, float* mean, 
 
 int pg_policy_logprob(pg_rollout* h, const pg_step_coef* coef, const float* x, const float* x_next,
                       const void* vel, const void* vel_ref, float* logp_out, float* kl_out, void* stream) {
+  TraceRange trace_range("pg_policy_logprob");
   if (!h || !coef || !x || !x_next || !vel || !logp_out) return PG_EINVAL;
   if (const int rc_dev = wrong_device(h)) return rc_dev;
   if ((vel_ref == nullptr) != (kl_out == nullptr)) return PG_EINVAL;
@@ -332,6 +351,7 @@ int pg_policy_logprob(pg_rollout* h, const pg_step_coef* coef, const float* x, c
 int pg_policy_objective(pg_rollout* h, int32_t n_steps, const float* logp_new, const float* logp_old,
                         const float* kl, const float* adv, float clip_eps, float beta, float* ratio,
                         float* dlogp, float* objective, void* stream) {
+  TraceRange trace_range("pg_policy_objective");
   if (!h || n_steps < 1 || !logp_new || !logp_old || !adv || !dlogp || !objective) return PG_EINVAL;
   if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (!(clip_eps >= 0.f) || !std::isfinite(beta)) return PG_EINVAL;
@@ -342,6 +362,7 @@ int pg_policy_objective(pg_rollout* h, int32_t n_steps, const float* logp_new, c
 int pg_policy_backward(pg_rollout* h, const pg_step_coef* coef, const float* x, const float* x_next,
                        const void* vel, const void* vel_ref, const float* dlogp, double dkl,
                        void* grad_vel, void* stream) {
+  TraceRange trace_range("pg_policy_backward");
   if (!h || !coef || !x || !x_next || !vel || !dlogp || !grad_vel) return PG_EINVAL;
   if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (!aligned16(x) || !aligned16(x_next) || !aligned16(vel) || !aligned16(vel_ref) ||
@@ -358,6 +379,7 @@ int pg_policy_backward(pg_rollout* h, const pg_step_coef* coef, const float* x, 
 int pg_ovf_select_batched(int32_t n_groups, int32_t n, int32_t k, const float* scores,
                           int32_t* keep_idx, float* kept_scores, float* adv, float adv_eps,
                           int32_t* status, void* stream) {
+  TraceRange trace_range("pg_ovf_select_batched");
   if (n_groups < 0 || n < 1 || n > PG_MAX_GROUP || k < 1 || k > n) return PG_EINVAL;
   if (!(adv_eps >= 0.f)) return PG_EINVAL;
   if (n_groups == 0) return PG_OK;
@@ -376,6 +398,7 @@ int pg_rollout_traj_ids(pg_rollout* h, int32_t* dst, void* stream) {
 }
 
 int pg_survivor_rows(pg_rollout* h, const int32_t* keep_idx_packed, int32_t* rows_out, void* stream) {
+  TraceRange trace_range("pg_survivor_rows");
   if (!h || !rows_out) return PG_EINVAL;
   if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (h->cfg.n_stages > 0 && !keep_idx_packed) return PG_EINVAL;
@@ -386,6 +409,7 @@ int pg_survivor_rows(pg_rollout* h, const int32_t* keep_idx_packed, int32_t* row
 
 int pg_survivor_logp(pg_rollout* h, const int32_t* rows, const float* logp_packed, float* logp_out,
                      void* stream) {
+  TraceRange trace_range("pg_survivor_logp");
   if (!h || !rows || !logp_packed || !logp_out) return PG_EINVAL;
   if (const int rc_dev = wrong_device(h)) return rc_dev;
   const int k_final = h->cfg.n_stages > 0 ? h->stage_keep.back() : h->cfg.n_expand;
@@ -395,6 +419,7 @@ int pg_survivor_logp(pg_rollout* h, const int32_t* rows, const float* logp_packe
 
 int pg_gather_rows(pg_rollout* h, const int32_t* rows, int32_t n_out, int32_t n_in, const void* src,
                    void* dst, size_t row_bytes, void* stream) {
+  TraceRange trace_range("pg_gather_rows");
   if (!h || n_out < 0 || n_in < 0 || row_bytes == 0) return PG_EINVAL;
   if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (n_out == 0) return PG_OK;
@@ -492,6 +517,7 @@ int pg_rollout_host(const pg_config* cfg, const pg_step_coef* step_coef,
                     const void* const* vel_steps, const float* const* stage_scores,
                     const float* final_rewards, float* x_final, float* logp, int32_t* keep_idx,
                     float* adv, int32_t* traj_id, void* workspace, size_t workspace_bytes) {
+  TraceRange trace_range("pg_rollout_host");
   int rc = validate_config(cfg);
   if (rc != PG_OK) return rc;
   if (!step_coef || !vel_steps || !workspace || !aligned16(workspace)) return PG_EINVAL;
@@ -650,6 +676,7 @@ int pg_rollout_run(pg_rollout* h, const pg_step_coef* step_coef, const pg_previe
                    const float* x0, const void* const* vel_steps, const float* const* stage_scores,
                    const float* final_rewards, void* workspace, size_t workspace_bytes,
                    pg_rollout_outputs* out, void* stream) {
+  TraceRange trace_range("pg_rollout_run");
   if (!h || !step_coef || !x0 || !vel_steps || !workspace || !out || !aligned16(workspace) ||
       !aligned16(x0))
     return PG_EINVAL;
