@@ -637,7 +637,7 @@ def main():
     ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="large", choices=["large", "sd3", "sd15", "tiny"])
+    ap.add_argument("--workload", default="large", choices=["large", "sd3", "sd15", "tiny", "pro-standard", "pro-flash", "pro-diffusion"])
     ap.add_argument("--groups", type=int, default=0,
                     help="prompt groups per GPU (default: the workload's own; smaller for profiling)")
     ap.add_argument("--no-e2e", action="store_true")

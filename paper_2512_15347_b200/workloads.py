@@ -89,6 +89,15 @@ WORKLOADS: Dict[str, Workload] = {
                     "normal", "external"),
     "large": Workload("large", 64, 64, ((2, 32), (5, 16), (8, 16)), 28, 16 * 128 * 128, 16, "bf16",
                       7, "normal", "preview"),
+    # the schedules of the paper's experimental settings (Section 6.1), 16 prompt groups each:
+    # Standard 48 -> 24 -> 12 and Flash 24 -> 16 -> 12 at steps {5, 7} of 10 on SD3-sized latents,
+    # and 48 -> 32 -> 8 at steps {30, 40} of 50 on SD-v1.4-sized latents
+    "pro-standard": Workload("pro-standard", 16, 48, ((5, 24), (7, 12)), 10, 16 * 128 * 128, 16, "bf16",
+                             11, "normal", "preview"),
+    "pro-flash": Workload("pro-flash", 16, 24, ((5, 16), (7, 12)), 10, 16 * 128 * 128, 16, "bf16",
+                          12, "normal", "preview"),
+    "pro-diffusion": Workload("pro-diffusion", 16, 48, ((30, 32), (40, 8)), 50, 4 * 64 * 64, 4, "bf16",
+                              13, "normal", "preview"),
 }
 
 # OVF selection microbenchmark: 4096 groups x 256 scores, keep 32.

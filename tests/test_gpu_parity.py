@@ -346,7 +346,9 @@ def test_rollout_matches_oracle(B, name):
     ro.close()
 
 
-@pytest.mark.parametrize("name,groups,elems", [("sd3", 4, 16384 + 8192 + 64), ("large", 3, 32768 + 4)])
+@pytest.mark.parametrize("name,groups,elems", [("sd3", 4, 16384 + 8192 + 64), ("large", 3, 32768 + 4),
+                                               ("pro-standard", 2, 8192 + 64), ("pro-flash", 3, 4096 + 4),
+                                               ("pro-diffusion", 2, 2048 + 36)])
 def test_scaled_rollout_matches_oracle(B, name, groups, elems):
     w = wl.scaled(wl.WORKLOADS[name], n_groups=groups, elems=elems)
     inp = U.SharedInputs(w)
