@@ -68,8 +68,8 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
 //   u1 = ((r0 >> 8) + 1) * 2^-24 in (0, 1],  u2 = (r1 >> 8) * 2^-24 in [0, 1)
 //   normals  a = sqrt(-2 ln u1) cos(2 pi u2),  b = sqrt(-2 ln u1) sin(2 pi u2)
 // Returned in factored form: radius = sqrt(-2 ln u1) and (c, s) = (cos, sin)(2 pi u2 - pi), so
-// that a = -radius * c and b = -radius * s (half-turn shift: the hardware sine / cosine are
-// evaluated on [-pi, pi), their most accurate range); the return value is -2 ln u1 = a^2 + b^2.
+// that a = -radius * c and b = -radius * s (half-turn shift: the hardware sine is evaluated on
+// [-pi, pi), its most accurate range); the return value is -2 ln u1 = a^2 + b^2.
 // The logarithm uses the hardware log2 except close to u1 = 1, where its absolute error would
 // dominate the small radius: there -2 ln(1 - w) is summed as a short series in w = 1 - u1 (exact
 // in fp32; truncation below 2e-8 relative for w < 2^-6).
@@ -88,9 +88,18 @@ __device__ __forceinline__ float box_muller(uint32_t r0, uint32_t r1, float& rad
   neg2ln = (w < 0.015625f) ? ser : neg2ln;
   asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(radius) : "f"(neg2ln));
   const float turn = fmaf((float)(r1 >> 8), 5.9604644775390625e-8f, -0.5f);  // u2 - 1/2, exact
+  // The cosine is taken as the sine of the angle a quarter turn further, wrapped back into
+  // [-1/2, 1/2) turns (all exact on the 24-bit grid).  The hardware sine's error is an odd
+  // function of the angle, so over the symmetric angle grid it averages to zero; the hardware
+  // cosine's error is even and does not (measured mean +5.8e-8, i.e. -7.2e-8 on every cosine
+  // normal) - small against the 2e-7 rms error of a draw, but a bias is what the mean of a long
+  // latent (the latent score) accumulates over many steps.
+  float turn_c = turn + 0.25f;
+  turn_c = turn_c >= 0.5f ? turn_c - 1.0f : turn_c;
   const float angle = 6.283185307179586f * turn;
+  const float angle_c = 6.283185307179586f * turn_c;
   asm("sin.approx.ftz.f32 %0, %1;" : "=f"(s) : "f"(angle));
-  asm("cos.approx.ftz.f32 %0, %1;" : "=f"(c) : "f"(angle));
+  asm("sin.approx.ftz.f32 %0, %1;" : "=f"(c) : "f"(angle_c));
   return neg2ln;
 }
 
@@ -266,7 +275,7 @@ int launch_step(int n_rows, int elems, int vel_dtype, const float* x_in, const v
                 int32_t* status = nullptr);
 
 int launch_score(int n_rows, int elems, int vel_dtype, const float* x, const void* vel,
-                 double p_x, double p_v, float* scores_out, float* preview_out,
+                 double p_x, double p_v, float* scores_out, void* preview_out, int preview_bf16,
                  RowScratch scratch, cudaStream_t stream, int forced_chunk_quads = 0);
 
 int launch_preview(int n_rows, int elems, int vel_dtype, const float* x, const void* vel, double p_x,
