@@ -165,6 +165,19 @@ int pg_score(pg_rollout *h, const pg_preview_coef *coef, const float *x, const v
              float *scores_out, float *preview_out, void *stream);
 
 /*
+ * Latent score and preview emission in one pass (Eq. "ode_lookahead_method" feeding Eq.
+ * "proxy_reward_method": the preview is what the VAE decoder and reward model outside this
+ * library consume, the score is the stand-in proxy reward).  Same as pg_score, but the preview
+ * is written in the type the consumer wants: preview_dtype PG_VEL_F32 (fp32) or PG_VEL_BF16 (bf16,
+ * rounded to nearest even from the fp32 preview), [n_active, d], 16-byte aligned; with bf16
+ * the pass moves 8 bytes per element (6 read, 2 written) instead of a 6-byte scoring pass plus an
+ * 8-byte pg_preview pass.  scores_out is reduced from the fp32 preview in either case, so it is
+ * bit-identical to pg_score's.  preview_out may be NULL (preview_dtype is then ignored).
+ */
+int pg_score_preview(pg_rollout *h, const pg_preview_coef *coef, const float *x, const void *vel,
+                     float *scores_out, void *preview_out, int32_t preview_dtype, void *stream);
+
+/*
  * Preview emission only (Eq. "ode_lookahead_method"): out[i] = p_x * x[i] + p_v * vel[i] for the
  * n_active rows, written as fp32 (out_dtype PG_VEL_F32) or bf16 rounded to nearest even
  * (PG_VEL_BF16), same [n_active, d] layout as the latents, for the VAE decoder and reward model

@@ -75,6 +75,7 @@ def lib() -> ctypes.CDLL:
     L.pg_step.argtypes = [vp, i32, ctypes.POINTER(StepCoef), vp, vp, vp, vp, vp, vp]
     L.pg_score.argtypes = [vp, ctypes.POINTER(PreviewCoef), vp, vp, vp, vp, vp]
     L.pg_preview.argtypes = [vp, ctypes.POINTER(PreviewCoef), vp, vp, vp, i32, vp]
+    L.pg_score_preview.argtypes = [vp, ctypes.POINTER(PreviewCoef), vp, vp, vp, vp, i32, vp]
     L.pg_prune_ovf.argtypes = [vp, i32, vp, vp, vp, vp, vp]
     L.pg_prune_uniform.argtypes = [vp, i32, vp, vp, vp]
     L.pg_group_stats.argtypes = [i32, i32, vp, ctypes.c_float, vp, vp, vp, vp]
@@ -110,7 +111,7 @@ def lib() -> ctypes.CDLL:
                  "pg_step", "pg_score", "pg_prune_ovf", "pg_compact", "pg_advantages",
                  "pg_ovf_select_batched", "pg_rollout_host", "pg_rollout_traj_ids",
                  "pg_philox_raw", "pg_normal_rows", "pg_score_static", "pg_policy_logprob",
-                 "pg_policy_objective", "pg_policy_backward", "pg_prune_uniform", "pg_group_stats", "pg_preview", "pg_rollout_run", "pg_rollout_restore"):
+                 "pg_policy_objective", "pg_policy_backward", "pg_prune_uniform", "pg_group_stats", "pg_preview", "pg_rollout_run", "pg_rollout_restore", "pg_score_preview"):
         getattr(L, name).restype = ctypes.c_int
     _lib = L
     return L
@@ -192,6 +193,14 @@ def score(h: int, coef, x, vel, scores_out, preview_out=None, stream=None) -> No
     c = PreviewCoef(*coef)
     _check(lib().pg_score(h, ctypes.byref(c), _p(x), _p(vel), _p(scores_out), _p(preview_out),
                           _stream(stream)), "pg_score")
+
+
+def score_preview(h: int, coef, x, vel, scores_out, preview_out, stream=None) -> None:
+    """Scores and the preview x_hat (fp32 or bf16 tensor, by its dtype) in one pass."""
+    c = PreviewCoef(*coef)
+    dt = VEL_BF16 if preview_out is not None and preview_out.dtype == torch.bfloat16 else VEL_F32
+    _check(lib().pg_score_preview(h, ctypes.byref(c), _p(x), _p(vel), _p(scores_out), _p(preview_out), dt,
+                                  _stream(stream)), "pg_score_preview")
 
 
 def preview(h: int, coef, x, vel, out, stream=None) -> None:

@@ -236,18 +236,25 @@ int pg_step(pg_rollout* h, int32_t step, const pg_step_coef* coef, const float* 
   return rc;
 }
 
-int pg_score(pg_rollout* h, const pg_preview_coef* coef, const float* x, const void* vel,
-             float* scores_out, float* preview_out, void* stream) {
+int pg_score_preview(pg_rollout* h, const pg_preview_coef* coef, const float* x, const void* vel,
+                     float* scores_out, void* preview_out, int32_t preview_dtype, void* stream) {
   TraceRange trace_range("pg_score");
   if (!h || !coef || !x || !scores_out) return PG_EINVAL;
   if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (!std::isfinite(coef->p_x) || !std::isfinite(coef->p_v)) return PG_EINVAL;
   if (coef->p_v != 0.0 && !vel) return PG_EINVAL;
+  if (preview_out && preview_dtype != PG_VEL_F32 && preview_dtype != PG_VEL_BF16) return PG_EINVAL;
   if (!aligned16(x) || !aligned16(vel) || !aligned16(preview_out)) return PG_EINVAL;
   const int rows = h->cfg.n_groups * h->k_cur;
   pg::RowScratch scratch{h->d_partials, h->d_tickets};
   return pg::launch_score(rows, h->cfg.elems, h->cfg.vel_dtype, x, vel, coef->p_x, coef->p_v,
-                          scores_out, preview_out, scratch, (cudaStream_t)stream);
+                          scores_out, preview_out, preview_dtype == PG_VEL_BF16, scratch,
+                          (cudaStream_t)stream);
+}
+
+int pg_score(pg_rollout* h, const pg_preview_coef* coef, const float* x, const void* vel,
+             float* scores_out, float* preview_out, void* stream) {
+  return pg_score_preview(h, coef, x, vel, scores_out, preview_out, PG_VEL_F32, stream);
 }
 
 int pg_preview(pg_rollout* h, const pg_preview_coef* coef, const float* x, const void* vel, void* out,

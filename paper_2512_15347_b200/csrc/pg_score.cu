@@ -1,7 +1,10 @@
 // ODE look-ahead preview and latent score (Eq. "ode_lookahead_method", Eq. "proxy_reward_method"):
-// x_hat = p_x * x + p_v * v, score = mean over the elements of x_hat.  Read-only streaming pass
-// (optionally emitting x_hat); the per-trajectory sum uses the same fixed-shape reduction as the
-// step kernel, so scores are reproducible from run to run.
+// x_hat = p_x * x + p_v * v, score = mean over the elements of x_hat.  Read-only streaming pass,
+// optionally emitting x_hat in the same pass as fp32 or as bf16 (what a decoder + reward model
+// placed between preview and selection consume: 8 bytes per element for score and preview
+// together instead of a 6-byte scoring pass plus an 8-byte emission pass); the per-trajectory sum
+// uses the same fixed-shape reduction as the step kernel, so scores are reproducible from run
+// to run.  The score is always reduced from the fp32 preview, whatever is emitted.
 #include "pg_common.cuh"
 
 namespace pg {
@@ -10,7 +13,7 @@ struct ScoreParams {
   const float* x;
   const void* vel;
   float* scores_out;
-  float* preview_out;
+  void* preview_out;
   float* partials;
   unsigned int* tickets;
   int quads_per_row;
@@ -33,17 +36,35 @@ template <typename T> struct VelRaw;
 template <> struct VelRaw<float> { using type = float4; };
 template <> struct VelRaw<__nv_bfloat16> { using type = uint2; };
 
+__device__ __forceinline__ void store_preview(float* out, size_t quad, const float4& v) {
+  __stcs(reinterpret_cast<float4*>(out) + quad, v);
+}
+__device__ __forceinline__ void store_preview(__nv_bfloat16* out, size_t quad, const float4& v) {
+  const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
+  const __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
+  uint2 w;
+  w.x = *reinterpret_cast<const unsigned int*>(&lo);
+  w.y = *reinterpret_cast<const unsigned int*>(&hi);
+  __stcs(reinterpret_cast<uint2*>(out) + quad, w);
+}
+
+// What the scoring pass writes besides the scores.
+enum : int { kEmitNone = 0, kEmitF32 = 1, kEmitBf16 = 2 };
+template <int kEmit> struct EmitType { using type = float; };
+template <> struct EmitType<kEmitBf16> { using type = __nv_bfloat16; };
+
 constexpr int kScoreUnroll = 4;   // quads per thread and iteration (loads of the next batch in flight)
 
-template <typename VelT, bool kUseVel, bool kEmit>
+template <typename VelT, bool kUseVel, int kEmit>
 __global__ void __launch_bounds__(kRowThreads)
 score_kernel(const __grid_constant__ ScoreParams p) {
   using Raw = typename VelRaw<VelT>::type;
+  using OutT = typename EmitType<kEmit>::type;
   const int row = blockIdx.x / p.chunks;
   const int chunk = blockIdx.x - row * p.chunks;
   const float4* x = reinterpret_cast<const float4*>(p.x) + (size_t)row * p.quads_per_row;
   const Raw* vel = reinterpret_cast<const Raw*>(p.vel) + (size_t)row * p.quads_per_row;
-  float4* prev = kEmit ? reinterpret_cast<float4*>(p.preview_out) + (size_t)row * p.quads_per_row : nullptr;
+  OutT* prev = kEmit ? reinterpret_cast<OutT*>(p.preview_out) + (size_t)row * p.quads_per_row * 4 : nullptr;
   const int q_begin = chunk * p.chunk_quads;
   const int q_end = min(q_begin + p.chunk_quads, p.quads_per_row);
 
@@ -82,7 +103,7 @@ score_kernel(const __grid_constant__ ScoreParams p) {
           h.w = fmaf(p.p_v, vf.w, h.w);
         }
         acc += (h.x + h.y) + (h.z + h.w);
-        if (kEmit) __stcs(prev + qq, h);
+        if (kEmit) store_preview(prev, (size_t)qq, h);
       }
     }
 #pragma unroll
@@ -95,21 +116,23 @@ score_kernel(const __grid_constant__ ScoreParams p) {
              [&](double sum) { p.scores_out[row] = (float)(sum * p.inv_d); });
 }
 
-template <typename VelT>
-static void dispatch_score(const ScoreParams& p, bool use_vel, bool emit, dim3 grid,
-                           cudaStream_t stream) {
+template <typename VelT, bool kUseVel>
+static void dispatch_score_emit(const ScoreParams& p, int emit, dim3 grid, cudaStream_t stream) {
   const dim3 block(kRowThreads);
-  if (use_vel) {
-    if (emit) score_kernel<VelT, true, true><<<grid, block, 0, stream>>>(p);
-    else      score_kernel<VelT, true, false><<<grid, block, 0, stream>>>(p);
-  } else {
-    if (emit) score_kernel<VelT, false, true><<<grid, block, 0, stream>>>(p);
-    else      score_kernel<VelT, false, false><<<grid, block, 0, stream>>>(p);
-  }
+  if (emit == kEmitBf16)     score_kernel<VelT, kUseVel, kEmitBf16><<<grid, block, 0, stream>>>(p);
+  else if (emit == kEmitF32) score_kernel<VelT, kUseVel, kEmitF32><<<grid, block, 0, stream>>>(p);
+  else                       score_kernel<VelT, kUseVel, kEmitNone><<<grid, block, 0, stream>>>(p);
+}
+
+template <typename VelT>
+static void dispatch_score(const ScoreParams& p, bool use_vel, int emit, dim3 grid,
+                           cudaStream_t stream) {
+  if (use_vel) dispatch_score_emit<VelT, true>(p, emit, grid, stream);
+  else         dispatch_score_emit<VelT, false>(p, emit, grid, stream);
 }
 
 int launch_score(int n_rows, int elems, int vel_dtype, const float* x, const void* vel,
-                 double p_x, double p_v, float* scores_out, float* preview_out,
+                 double p_x, double p_v, float* scores_out, void* preview_out, int preview_bf16,
                  RowScratch scratch, cudaStream_t stream, int forced_chunk_quads) {
   if (n_rows == 0) return PG_OK;
   const RowGeometry geo = row_geometry(n_rows, elems, forced_chunk_quads);
@@ -130,25 +153,15 @@ int launch_score(int n_rows, int elems, int vel_dtype, const float* x, const voi
   if (blocks > 0x7FFFFFFFLL) return PG_EINVAL;
   const dim3 grid((unsigned)blocks);
   const bool use_vel = (p_v != 0.0);
-  if (vel_dtype == PG_VEL_BF16) dispatch_score<__nv_bfloat16>(p, use_vel, preview_out != nullptr, grid, stream);
-  else                          dispatch_score<float>(p, use_vel, preview_out != nullptr, grid, stream);
+  const int emit = !preview_out ? kEmitNone : (preview_bf16 ? kEmitBf16 : kEmitF32);
+  if (vel_dtype == PG_VEL_BF16) dispatch_score<__nv_bfloat16>(p, use_vel, emit, grid, stream);
+  else                          dispatch_score<float>(p, use_vel, emit, grid, stream);
   PG_LAUNCH_CHECK();
   return PG_OK;
 }
 
 // ---------------------------------------------------------------- preview emission only
 
-__device__ __forceinline__ void store_preview(float* out, size_t quad, const float4& v) {
-  __stcs(reinterpret_cast<float4*>(out) + quad, v);
-}
-__device__ __forceinline__ void store_preview(__nv_bfloat16* out, size_t quad, const float4& v) {
-  const __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y);
-  const __nv_bfloat162 hi = __floats2bfloat162_rn(v.z, v.w);
-  uint2 w;
-  w.x = *reinterpret_cast<const unsigned int*>(&lo);
-  w.y = *reinterpret_cast<const unsigned int*>(&hi);
-  __stcs(reinterpret_cast<uint2*>(out) + quad, w);
-}
 
 // x_hat = p_x x + p_v v written in fp32 or bf16 (for a decoder that follows); no reduction.
 template <typename VelT, typename OutT>

@@ -74,5 +74,5 @@ extern "C" int pg_score_static(int32_t n_rows, int32_t elems, int32_t vel_dtype,
   PG_CUDA(cudaMemsetAsync(s->tickets, 0, (size_t)n_rows * sizeof(unsigned int), st));
   pg::RowScratch scratch{s->partials, s->tickets};
   return pg::launch_score(n_rows, elems, vel_dtype, x, vel, coef->p_x, coef->p_v, scores_out,
-                          nullptr, scratch, st, kStaticChunkQuads);
+                          nullptr, 0, scratch, st, kStaticChunkQuads);
 }
