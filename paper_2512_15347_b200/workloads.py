@@ -13,12 +13,15 @@ settings of Section 6.1).
 """
 from __future__ import annotations
 
+import functools
 import math
 from dataclasses import dataclass
 from typing import Dict, List, Optional, Tuple
 
 import numpy as np
 import torch
+
+from . import schedules as sch
 
 
 @dataclass(frozen=True)
@@ -32,10 +35,12 @@ class Workload:
     channels: int
     vel_dtype: str                # "fp32" | "bf16"
     seed: int
-    velocity: str                 # "affine" (config 1) | "normal" (fresh N(0,1) per step)
+    velocity: str                 # "affine" (config 1) | "normal" (fresh N(0,1) per step) | "eps"
     scores: str                   # "preview" | "external"
     sigma: float = 0.7            # noise_std = sigma * sqrt(dt)
     adv_eps: float = 1e-6
+    coef: str = "rf-drift"        # source of the per-step coefficients, see step_coef()
+    eta: float = 1.0              # stochasticity of the diffusion samplers ("ddim", "vp-em")
 
     @property
     def final_keep(self) -> int:
@@ -73,13 +78,59 @@ class Workload:
         return sum(self.n_groups * self.rows_before(s) for s, _ in self.stages)
 
     def step_coef(self, step: int) -> Tuple[float, float, float]:
-        """(c_x, c_v, noise_std): drift = the supplied prediction, uniform dt = 1/T."""
+        """(c_x, c_v, noise_std) of SDE step `step` on the uniform grid t_s = s/T.
+
+        coef = "rf-drift": drift = the supplied prediction (c_x = 1, c_v = dt);
+        "rf-sde": rectified flow with the score-corrected drift of Eq. rf_sde_general;
+        "ddim": epsilon-prediction diffusion, the T-step DDIM / ancestral sampler (stochasticity
+        eta) over the 1000-step linear-beta schedule; its last step lands on the clean sample and
+        is deterministic (noise_std = 0);
+        "vp-em": Euler-Maruyama of Eq. dm_sde for the continuous variance-preserving diffusion
+        with beta(tau) = 0.1 + 19.9 tau, tau = 1 - s/T the noise-level time."""
         dt = 1.0 / self.n_steps
-        return 1.0, dt, self.sigma * math.sqrt(dt)
+        if self.coef == "rf-drift":
+            return sch.rf_drift_coef(dt, self.sigma)
+        if self.coef == "rf-sde":
+            return sch.rf_sde_coef(step * dt, dt, self.sigma)
+        if self.coef == "ddim":
+            return _ddim_table(self.n_steps, self.eta)[step]
+        if self.coef == "vp-em":
+            beta, sigma_bar = _vp_continuous(1.0 - step * dt)
+            return sch.vp_em_coef(beta, sigma_bar, dt, self.eta)
+        raise ValueError(f"unknown coefficient source {self.coef!r}")
 
     def preview_coef(self, step: int) -> Tuple[float, float]:
-        """(p_x, p_v): one Euler step of the probability-flow ODE over the remaining time."""
-        return 1.0, 1.0 - step / self.n_steps
+        """(p_x, p_v) of the look-ahead preview at step `step` (Eq. ode_lookahead_method): one Euler
+        step of the probability-flow ODE over the remaining time for the rectified-flow sources and
+        "vp-em", the clean-sample estimate (x - sigma_t eps) / alpha_t for "ddim"."""
+        t = step / self.n_steps
+        if self.coef in ("rf-drift", "rf-sde"):
+            return sch.rf_preview_coef(t)
+        if self.coef == "ddim":
+            alpha, sigma = _vp_table()
+            i = round((len(alpha) - 1) * (1.0 - t))
+            return sch.x0_preview_coef(alpha[i], sigma[i])
+        if self.coef == "vp-em":
+            beta, sigma_bar = _vp_continuous(1.0 - t)
+            return sch.vp_euler_preview_coef(beta, sigma_bar, 1.0 - t)
+        raise ValueError(f"unknown coefficient source {self.coef!r}")
+
+
+@functools.lru_cache(maxsize=None)
+def _vp_table():
+    return sch.vp_linear_schedule()
+
+
+@functools.lru_cache(maxsize=None)
+def _ddim_table(n_steps: int, eta: float):
+    return sch.ddim_schedule(n_steps, eta)
+
+
+def _vp_continuous(tau: float) -> Tuple[float, float]:
+    """(beta(tau), sigma_bar(tau)) of the continuous linear-beta variance-preserving diffusion."""
+    b0, b1 = 0.1, 20.0
+    integral = b0 * tau + 0.5 * (b1 - b0) * tau * tau
+    return b0 + (b1 - b0) * tau, math.sqrt(-math.expm1(-integral))
 
 
 WORKLOADS: Dict[str, Workload] = {
@@ -96,8 +147,10 @@ WORKLOADS: Dict[str, Workload] = {
                              11, "normal", "preview"),
     "pro-flash": Workload("pro-flash", 16, 24, ((5, 16), (7, 12)), 10, 16 * 128 * 128, 16, "bf16",
                           12, "normal", "preview"),
-    "pro-diffusion": Workload("pro-diffusion", 16, 48, ((30, 32), (40, 8)), 50, 4 * 64 * 64, 4, "bf16",
-                              13, "normal", "preview"),
+    # (epsilon-prediction diffusion backbone: DDIM / ancestral coefficients, clean-sample preview,
+    # predictions correlated with the latent as a noise-prediction network's are)
+    "pro-diffusion": Workload("pro-diffusion", 16, 48, ((30, 32), (40, 8)), 50, 4 * 64 * 64, 4, "fp32",
+                              13, "eps", "preview", coef="ddim", eta=1.0),
 }
 
 # OVF selection microbenchmark: 4096 groups x 256 scores, keep 32.
@@ -129,9 +182,39 @@ def initial_latents(w: Workload, device="cpu") -> torch.Tensor:
 
 def normal_velocity(w: Workload, step: int, rows: int, device="cpu") -> torch.Tensor:
     """Stand-in network prediction for one step: fresh N(0,1), in the workload's dtype."""
-    v = torch.randn(rows, w.elems, generator=_gen(device, w.seed, 202, step), device=device,
-                    dtype=torch.float32)
+    v = normal_noise(w, step, rows, device)
     return v.to(torch.bfloat16) if w.vel_dtype == "bf16" else v
+
+
+def normal_noise(w: Workload, step: int, rows: int, device="cpu") -> torch.Tensor:
+    """The fp32 N(0,1) draws behind normal_velocity (before any rounding to bf16)."""
+    return torch.randn(rows, w.elems, generator=_gen(device, w.seed, 202, step), device=device,
+                       dtype=torch.float32)
+
+
+def eps_mix(w: Workload, step: int) -> Tuple[float, float]:
+    """(a, b) of the stand-in noise-prediction network at step `step`: eps_hat = a x + b z.
+
+    For unit-variance Gaussian data under x_t = alpha_t x_1 + sigma_t eps the exact noise
+    prediction is E[eps | x_t] = sigma_t x_t; the stand-in adds an independent error term
+    alpha_t z, z ~ N(0, I), so that eps_hat is N(0, 1) per element like the target and correlated
+    with the latent like a real network's output (an uncorrelated prediction would let the
+    epsilon-prediction samplers, whose c_x exceeds 1, blow the latents up)."""
+    t = step / w.n_steps
+    if w.coef == "ddim":
+        alpha, sigma = _vp_table()
+        i = round((len(alpha) - 1) * (1.0 - t))
+        return sigma[i], alpha[i]
+    _, sigma_bar = _vp_continuous(1.0 - t)
+    return sigma_bar, math.sqrt(max(0.0, 1.0 - sigma_bar * sigma_bar))
+
+
+def eps_velocity(x: torch.Tensor, z: torch.Tensor, a: float, b: float, vel_dtype: str) -> torch.Tensor:
+    """eps_hat = a x + b z as three separately rounded fp32 operations (identical on CPU and GPU),
+    then rounded to the workload's prediction dtype."""
+    v = x * a
+    v += z * b
+    return v.to(torch.bfloat16) if vel_dtype == "bf16" else v
 
 
 def affine_field(w: Workload, device="cpu") -> Tuple[torch.Tensor, torch.Tensor]:

@@ -330,7 +330,7 @@ def test_advantages_match_oracle(B, G, K):
 
 # ------------------------------------------------------------------ whole rollouts
 
-@pytest.mark.parametrize("name", ["tiny", "sd15"])
+@pytest.mark.parametrize("name", ["tiny", "sd15", "pro-diffusion"])
 def test_rollout_matches_oracle(B, name):
     w = wl.WORKLOADS[name]
     inp = U.SharedInputs(w)
@@ -545,6 +545,32 @@ def test_out_of_sequence_calls_are_refused(B):
     finally:
         torch.cuda.synchronize()
         B.rollout_destroy(h)
+
+
+@pytest.mark.parametrize("name,coef,eta,groups,elems", [
+    ("pro-diffusion", "ddim", 0.5, 3, 16384),          # DDIM with partial stochasticity, full-length SD latents
+    ("pro-diffusion", "vp-em", 1.0, 2, 8192 + 36),     # Euler-Maruyama of the VP reverse SDE
+    ("pro-standard", "rf-sde", 1.0, 2, 32768 + 4),     # rectified flow with the score-corrected drift
+    ("large", "ddim", 1.0, 2, 65536 + 8),              # early checkpoints: large preview coefficients
+])
+def test_rollout_under_other_backbones_matches_oracle(B, name, coef, eta, groups, elems):
+    """Coefficients of the diffusion branch (Eq. dm_sde, epsilon prediction: c_x != 1, c_v < 0, a
+    noise level that changes from step to step, clean-sample or probability-flow previews) and of
+    the score-corrected rectified flow cross the C ABI and give the oracle's rollout."""
+    from dataclasses import replace
+    w = replace(wl.scaled(wl.WORKLOADS[name], n_groups=groups, elems=elems), coef=coef, eta=eta)
+    if coef != "rf-sde":
+        w = replace(w, velocity="eps", vel_dtype="fp32")     # stand-in noise-prediction network in the loop
+    c = [w.step_coef(s) for s in range(w.n_steps)]
+    assert all(abs(cx - 1.0) > 1e-3 for cx, _, _ in c)              # never the unit-c_x fast path
+    if coef != "rf-sde":
+        assert all(cv < 0 for _, cv, _ in c) and len({ns for _, _, ns in c}) == w.n_steps
+    inp = U.SharedInputs(w)
+    ref = U.run_oracle(w, inp)
+    ro, out = U.run_gpu(w, inp)
+    U.compare_rollouts(w, ref, out)
+    assert B.rollout_status(ro.h) == (groups * w.final_keep, w.n_steps, 0)
+    ro.close()
 
 
 # ------------------------------------------------------------------ edge schedules
@@ -778,6 +804,45 @@ def test_preview_emission_matches_oracle(B, bf16_vel, d):
         # bf16: 8 significant bits, round to nearest
         assert U.latent_err(out16.float().cpu().numpy(), ref) <= 2.0 ** -8
         assert torch.equal(out16, out32.to(torch.bfloat16))
+    finally:
+        torch.cuda.synchronize()
+        B.rollout_destroy(h)
+
+
+@pytest.mark.parametrize("bf16_vel", [False, True])
+@pytest.mark.parametrize("d", [4, 1000, 3 * 8192 + 20, 262144])
+def test_score_with_bf16_preview_in_one_pass_matches_oracle(B, bf16_vel, d):
+    """pg_score_preview: the scores are pg_score's bit for bit and the oracle's within the score
+    tolerance; the bf16 preview is the fp32 preview rounded to nearest even, i.e. the oracle's
+    preview to 8 significant bits."""
+    n_groups, n0 = 3, 4
+    n = n_groups * n0
+    rng = np.random.default_rng(d + 7 * bf16_vel)
+    x = rng.standard_normal((n, d)).astype(np.float32) - 0.2
+    vt = torch.from_numpy(rng.standard_normal((n, d)).astype(np.float32))
+    vt = vt.to(torch.bfloat16) if bf16_vel else vt
+    v = wl.as_numpy_velocity(vt)
+    h, _ = _handle(B, n_groups, n0, d, bf16=bf16_vel)
+    try:
+        coef = (2.27, -2.04)          # a clean-sample preview of the diffusion branch
+        ref, ref_prev = oracle.score(x, v, *coef, want_preview=True)
+        x_dev, v_dev = U.to_dev(x), U.vel_to_dev(v)
+        sc16, sc32, sc0 = (torch.empty(n, device="cuda") for _ in range(3))
+        out16 = torch.full((n, d), float("nan"), device="cuda", dtype=torch.bfloat16)
+        out32 = torch.empty(n, d, device="cuda")
+        B.score_preview(h, coef, x_dev, v_dev, sc16, out16)
+        B.score_preview(h, coef, x_dev, v_dev, sc32, out32)
+        B.score(h, coef, x_dev, v_dev, sc0)
+        assert torch.equal(sc16, sc0) and torch.equal(sc32, sc0)
+        # the preview has rms ~3: the score tolerance scales with it
+        assert np.abs(sc16.cpu().numpy() - ref).max() <= 3e-6
+        assert U.latent_err(out32.cpu().numpy(), ref_prev) <= 1e-6
+        assert torch.equal(out16, out32.to(torch.bfloat16))
+        assert U.latent_err(out16.float().cpu().numpy(), ref_prev) <= 2.0 ** -8
+        # without a velocity term
+        B.score_preview(h, (0.5, 0.0), x_dev, None, sc16, out16)
+        assert torch.equal(out16, (0.5 * x_dev).to(torch.bfloat16))
+        assert np.abs(sc16.cpu().numpy() - 0.5 * x.astype(np.float64).mean(axis=1)).max() <= 1e-6
     finally:
         torch.cuda.synchronize()
         B.rollout_destroy(h)

@@ -65,6 +65,10 @@ class SharedInputs:
         if w.velocity == "affine":
             a, b = self.affine
             return wl.affine_velocity(torch.from_numpy(x), a, b).numpy()
+        if w.velocity == "eps":
+            z = wl.normal_noise(w, step, x.shape[0])
+            a, b = wl.eps_mix(w, step)
+            return wl.as_numpy_velocity(wl.eps_velocity(torch.from_numpy(x), z, a, b, w.vel_dtype))
         if step not in self._vel:
             rows = w.n_groups * w.rows_before(step)
             self._vel[step] = wl.as_numpy_velocity(wl.normal_velocity(w, step, rows))
@@ -77,6 +81,16 @@ class SharedInputs:
         if w.velocity == "affine":
             a, b = self.affine
             return wl.affine_velocity(x, a.cuda(), b.cuda())
+        if w.velocity == "eps":
+            # the stand-in network runs on the device's own latents, as the affine field does (a
+            # closed loop on either side: the epsilon-prediction samplers amplify whatever is not
+            # fed back, c_x > 1).  fp32 predictions only: with bf16 a last-bit difference between
+            # the two latent tensors could flip a rounding of the prediction and show up as a
+            # 0.4 % difference in that element.
+            assert w.vel_dtype == "fp32"
+            z = wl.normal_noise(w, step, x.shape[0]).cuda()
+            a, b = wl.eps_mix(w, step)
+            return wl.eps_velocity(x, z, a, b, w.vel_dtype)
         return vel_to_dev(self.vel_numpy(step, np.empty((x.shape[0], 0))))
 
 
