@@ -121,6 +121,10 @@ class OracleSample:
         if w.velocity == "affine":
             a, b = wl.affine_field(sw)
             self.velocity = lambda s, x, traj: wl.affine_velocity(torch.from_numpy(x), a, b).numpy()
+        elif w.velocity == "eps":
+            zs = [wl.normal_noise(sw, s, groups * w.rows_before(s)) for s in range(w.n_steps)]
+            self.velocity = lambda s, x, traj: wl.as_numpy_velocity(
+                wl.eps_velocity(torch.from_numpy(x), zs[s], *wl.eps_mix(sw, s), sw.vel_dtype))
         else:
             vels = [wl.as_numpy_velocity(wl.normal_velocity(sw, s, groups * w.rows_before(s)))
                     for s in range(w.n_steps)]
@@ -205,6 +209,11 @@ def _gpu_inputs(w, wr, ro, dev, rank):
     if w.velocity == "affine":
         a_c, b_c = wl.affine_field(wr, device=dev)
         velocity = lambda s, x: wl.affine_velocity(x, a_c, b_c)   # stand-in network, inside the timing
+    elif w.velocity == "eps":
+        zs = [wl.normal_noise(wr, s, w.n_groups * w.rows_before(s), device=dev) for s in range(w.n_steps)]
+        mix = [wl.eps_mix(wr, s) for s in range(w.n_steps)]
+        # stand-in noise-prediction network (3 torch ops per step), inside the timing
+        velocity = lambda s, x: wl.eps_velocity(x, zs[s], *mix[s], wr.vel_dtype)
     else:
         vels = [wl.normal_velocity(wr, s, w.n_groups * w.rows_before(s), device=dev)
                 for s in range(w.n_steps)]
@@ -270,7 +279,7 @@ def _other_workload(name, dev, reps, peak):
         gms = a.elapsed_time(b) / reps
         graph = {"ms_per_rollout": gms, "latent_steps_per_s": w.traj_steps / (gms * 1e-3)}
         del nat
-    elif w.velocity == "affine" and w.scores == "preview":
+    elif w.velocity in ("affine", "eps") and w.scores == "preview":
         # predictions depend on the latents: the step-by-step driver with the stand-in network's
         # torch ops recorded into one CUDA graph
         from paper_2512_15347_b200.rollout import GraphedRollout
@@ -284,7 +293,7 @@ def _other_workload(name, dev, reps, peak):
         torch.cuda.synchronize()
         gms = a.elapsed_time(b) / reps
         graph = {"ms_per_rollout": gms, "latent_steps_per_s": w.traj_steps / (gms * 1e-3),
-                 "note": "stand-in network (2 torch ops per step) inside the graph"}
+                 "note": "stand-in network (a few torch ops per step) inside the graph"}
         del gr
     ro.close()
     return {"ms_per_rollout": ms, "cuda_graph_replay": graph, "latent_steps_per_s": w.traj_steps / (ms * 1e-3), "step_gbs": step_gbs,
@@ -341,8 +350,13 @@ def run_ours(args):
     wr = replace(w, seed=w.seed + 1000 * rank)
 
     dt = torch.bfloat16 if w.vel_dtype == "bf16" else torch.float32
-    ro = Rollout(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, dt, adv_eps=w.adv_eps,
-                 group_offset=sharding.weak_shard(w.n_groups, rank)[0])
+    # weak scaling: world x n_groups groups dealt out in contiguous blocks, this rank's block
+    # starting at group rank * n_groups (its handle gets that offset, so trajectory ids are global)
+    from paper_2512_15347_b200.sharded import ShardedRollout
+    sr = ShardedRollout(world * w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, dt,
+                        adv_eps=w.adv_eps, dist=dist)
+    assert (sr.first, sr.count) == sharding.weak_shard(w.n_groups, rank)
+    ro = sr.local
     x0, velocity, ext, fin, vels = _gpu_inputs(w, wr, ro, dev, rank)
     torch.cuda.synchronize()
 
@@ -367,7 +381,7 @@ def run_ours(args):
     ev0.record()
     for _ in range(args.steps):
         tr = []
-        one_rollout(trace=tr)
+        last_out = one_rollout(trace=tr)
         traces.append(tr)
     ev1.record()
     torch.cuda.synchronize()
@@ -375,9 +389,15 @@ def run_ours(args):
     launches = B.launch_count() - launches0
     clocks = sampler.stop(t_wall0, t_wall1)
     total_ms = ev0.elapsed_time(ev1)
+    gathered = None
     if dist is not None:
         dist.barrier()
-        total_ms = sharding.max_over_ranks(total_ms, dist, dev)
+        total_ms = sr.max_over_ranks(total_ms, dev)
+        # outside the timed region: the per-group results of all ranks in global group order
+        res = sr.gather(last_out, device=dev)
+        gathered = {"groups": int(res.mean.numel()), "survivors": int(res.traj_id.numel()),
+                    "shards": res.shards,
+                    "adv_abs_group_mean_max": float(res.adv.view(res.mean.numel(), -1).mean(dim=1).abs().max())}
 
     # per-kernel device times from the events recorded inside the timed region
     kinds = {}
@@ -550,8 +570,10 @@ def run_ours(args):
                 "score_gbs": score_gbs, "prune_stage_gbs": prune_stage_gbs,
                 "hbm_gbs_whole_rollout": (step_bytes + (score_bytes if score_gbs else 0)) / (total_ms * 1e-3) / 1e9,
                 "ovf_microbench": ovf, "drivers": drivers, "policy_update": policy, "other_kernels": other, "other_workloads": others, "e2e": e2e, "cpu_baseline": cpu_base}
+        if gathered is not None:
+            line["gathered"] = gathered
         print(json.dumps(line))
-    ro.close()
+    sr.close()
     if dist is not None:
         dist.destroy_process_group()
     return 0

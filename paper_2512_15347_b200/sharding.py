@@ -33,13 +33,29 @@ def max_over_ranks(value: float, dist=None, device=None) -> float:
     return float(t.item())
 
 
-def all_gather_groups(t, dist=None):
+def all_gather_groups(t, dist=None, group=None):
     """Concatenates a per-group (or per-trajectory) tensor over ranks in rank order, i.e. in global
-    group order for contiguous shards of equal size.  The only collective the sharded rollout can
-    need: a few KB of advantages / statistics when one rank wants the whole batch."""
-    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+    group order for contiguous shards.  Shards may differ in their first dimension (group_shard
+    hands the first ranks one group more; a rank may even hold nothing): the lengths are exchanged
+    first, every rank pads to the longest, and the padding is cut away after the gather.  The only
+    collective the sharded rollout can need: a few KB of advantages / statistics when one rank
+    wants the whole batch."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size(group) == 1:
         return t
     import torch
-    parts = [torch.empty_like(t) for _ in range(dist.get_world_size())]
-    dist.all_gather(parts, t.contiguous())
-    return torch.cat(parts, dim=0)
+    world = dist.get_world_size(group)
+    t = t.contiguous()
+    n_local = torch.tensor([t.shape[0]], dtype=torch.int64, device=t.device)
+    lengths = [torch.empty_like(n_local) for _ in range(world)]
+    dist.all_gather(lengths, n_local, group=group)
+    lengths = [int(v.item()) for v in lengths]
+    longest = max(lengths)
+    if longest == 0:
+        return t
+    padded = t
+    if t.shape[0] < longest:
+        padded = torch.zeros((longest,) + tuple(t.shape[1:]), dtype=t.dtype, device=t.device)
+        padded[: t.shape[0]] = t
+    parts = [torch.empty_like(padded) for _ in range(world)]
+    dist.all_gather(parts, padded, group=group)
+    return torch.cat([p[:n] for p, n in zip(parts, lengths)], dim=0)

@@ -61,3 +61,39 @@ def test_gpu_arm_prints_roofline_baseline_and_end_to_end():
     assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0
     assert e["value"] != d["value"]
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
+
+
+def _torchrun(args, timeout=600):
+    """One rank under the distributed launcher (rendezvous on 127.0.0.1): the process-group set-up,
+    the build barrier, the max-over-ranks reduction and the gather all execute, on one GPU."""
+    port = 23000 + os.getpid() % 4000
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "1",
+           "--master-addr", "127.0.0.1", "--master-port", str(port)] + args
+    env = dict(os.environ, NCCL_NVLS_ENABLE="0")
+    p = subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=timeout)
+    assert p.returncode == 0, (p.stdout[-1500:], p.stderr[-2500:])
+    return [ln for ln in p.stdout.splitlines() if ln.strip().startswith("{")]
+
+
+@pytest.mark.gpu
+def test_gpu_arm_under_the_distributed_launcher():
+    lines = _torchrun(["bench.py", "--gpus", "1", "--workload", "sd15", "--steps", "2", "--warmup", "3",
+                       "--no-e2e", "--no-cpu-baseline"])
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 1 and d["value"] > 0 and d["gpu_launches"] > 0
+    g = d["gathered"]                     # only present when a process group exists
+    assert g["groups"] == 8 and g["survivors"] == 8 * 12 and g["shards"] == [[0, 8]]
+    assert g["adv_abs_group_mean_max"] < 1e-5
+
+
+@pytest.mark.gpu
+def test_sharded_launcher_runs_and_gathers():
+    lines = _torchrun(["-m", "paper_2512_15347_b200.sharded", "--workload", "sd15", "--groups", "5",
+                       "--reps", "2"])
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["ranks"] == 1 and d["groups"] == 5 and d["shards"] == [[0, 5]] and d["survivors"] == 5 * 12
+    assert d["latent_steps_per_s"] > 0 and d["adv_abs_mean_per_group_max"] < 1e-5
+    # trajectory ids are global ids of 5 groups x 24 trajectories
+    assert 0 < d["traj_id_checksum"] < 5 * 12 * 5 * 24
