@@ -303,6 +303,68 @@ def _other_workload(name, dev, reps, peak):
 
 
 
+LAUNCH_ROWS = (192, 384, 768, 1024, 2048, 4096)
+
+
+def launch_size_table(B, x_a, x_b, vel, elems, peak, rows_list=LAUNCH_ROWS, reps=24):
+    """Step and score launches of the streaming shape (d = `elems`, bf16 predictions) by row count:
+    device time per launch and algorithmic GB/s, measured two ways - `stream`: `reps` launches
+    enqueued back to back between one pair of CUDA events (how a rollout issues them; successive
+    launches use different rows of the buffers, so nothing is served from L2), and `isolated`: the
+    median of single launches, each between its own pair of events on an idle GPU.  x_a, x_b:
+    fp32 [>= max rows, d] (read / written), vel bf16 [>= max rows, d]."""
+    import torch
+    out = {"elems": elems, "reps": reps, "bytes_per_element": {"step": 10, "score": 6}, "rows": {}}
+    cap = min(x_a.shape[0], vel.shape[0])
+    lp = torch.empty(cap, device=x_a.device)
+    sc = torch.empty(cap, device=x_a.device)
+    for rows in rows_list:
+        if rows > cap:
+            continue
+        h = B.rollout_init(B.make_config(rows, 1, elems, 1 << 30, [], 3, B.VEL_BF16))
+        nxt = [0]
+        span = cap - rows + 1
+
+        def step(i):
+            o = (i * rows) % span
+            B.step(h, nxt[0], (1.0, 0.04, 0.13), x_a[o:o + rows], vel[o:o + rows], None, x_b[o:o + rows], lp)
+            nxt[0] += 1
+
+        def score(i):
+            o = (i * rows) % span
+            B.score(h, (1.0, 0.5), x_a[o:o + rows], vel[o:o + rows], sc)
+
+        entry = {}
+        for name, fn, bpe in (("step", step, 10), ("score", score, 6)):
+            for i in range(3):
+                fn(i)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(reps):
+                fn(i)
+            b.record()
+            torch.cuda.synchronize()
+            stream_us = a.elapsed_time(b) / reps * 1e3
+            singles = []
+            for i in range(reps):
+                a.record()
+                fn(i)
+                b.record()
+                torch.cuda.synchronize()
+                singles.append(a.elapsed_time(b) * 1e3)
+            singles.sort()
+            iso_us = singles[len(singles) // 2]
+            nbytes = rows * (elems * bpe + 4)
+            entry[name] = {"stream_us": stream_us, "stream_gbs": nbytes / stream_us / 1e3,
+                           "stream_frac": nbytes / stream_us / 1e3 / peak,
+                           "isolated_us": iso_us, "isolated_gbs": nbytes / iso_us / 1e3}
+        out["rows"][str(rows)] = entry
+        torch.cuda.synchronize()
+        B.rollout_destroy(h)
+    return out
+
+
 def run_ours(args):
     import torch
     from paper_2512_15347_b200 import binding as B
@@ -533,6 +595,11 @@ def run_ours(args):
                  "note": "pg_compact gathers the first stage's survivors (fp32 rows); pg_preview writes "
                          "the bf16 look-ahead latent for an external decoder"}
 
+    # step / score launches by row count on the streaming shape
+    by_rows = None
+    if rank == 0 and w.vel_dtype == "bf16" and w.velocity == "normal" and w.elems * w.n_groups * w.n_expand * 4 > 1e9:
+        by_rows = launch_size_table(B, ro.x[0], ro.x[1], vels[0], w.elems, peak)
+
     # the three smaller workloads, same driver (secondary lines; the bench line is the large one)
     others = None
     if rank == 0 and world == 1 and args.workload == "large" and not args.groups and not args.no_others:
@@ -569,7 +636,7 @@ def run_ours(args):
                                 v["launches"] // args.steps} for k, v in kinds.items()},
                 "score_gbs": score_gbs, "prune_stage_gbs": prune_stage_gbs,
                 "hbm_gbs_whole_rollout": (step_bytes + (score_bytes if score_gbs else 0)) / (total_ms * 1e-3) / 1e9,
-                "ovf_microbench": ovf, "drivers": drivers, "policy_update": policy, "other_kernels": other, "other_workloads": others, "e2e": e2e, "cpu_baseline": cpu_base}
+                "ovf_microbench": ovf, "drivers": drivers, "policy_update": policy, "other_kernels": other, "launch_size_table": by_rows, "other_workloads": others, "e2e": e2e, "cpu_baseline": cpu_base}
         if gathered is not None:
             line["gathered"] = gathered
         print(json.dumps(line))

@@ -144,34 +144,28 @@ __device__ __forceinline__ double warp_sum(double v) {
 #endif  // __CUDACC__
 
 // ---------------------------------------------------------------- launch geometry
-// Row-streaming kernels (step, score): a CTA of kRowThreads threads handles one chunk of one
-// row and contributes one partial sum, so a row owns `chunks` partial slots.  Chunks are
-// 2048 or 4096 quads (4-element groups): shorter chunks pay the end-of-CTA reduction (a barrier,
-// a fence and an atomic) too often, longer ones measured 1 % slower in back-to-back launches and
-// 4 % slower in isolated ones (fewer, longer CTAs drain less evenly at the end of a launch).
+// Row-streaming kernels (step, score, policy log-prob): a CTA of kRowThreads threads handles one
+// chunk of one row and contributes one partial sum, so a row owns `chunks` partial slots.  A chunk
+// is 2048 quads (4-element groups) whatever the number of rows, so the shape of a row's reduction
+// depends on the row length alone: a trajectory gets the same bits in a batch of any size, on any
+// shard.  Measured on 192 ... 4096 rows of 65536 quads, back-to-back launches: 1024-quad chunks
+// are 10 % slower (a CTA's launch, its first unoverlapped loads and its end-of-CTA barrier, fence
+// and atomic come twice as often), 3072- and 4096-quad chunks 1 - 3 % slower (fewer, longer CTAs
+// drain less evenly at the end of a launch).
 constexpr int kRowThreads = 256;
 constexpr int kRowWarps = kRowThreads / 32;
-constexpr int kMinChunkQuads = 2048;                   // 8192 elements
-constexpr int kMaxChunkQuads = 4096;                   // 16384 elements
-constexpr long long kWantedCtas = 148LL * 4 * 16;      // CTAs for ~16 waves at 4 CTAs per SM
+constexpr int kChunkQuads = 2048;                      // 8192 elements per CTA
 
 struct RowGeometry {
   int chunk_quads;   // quads per CTA
   int chunks;        // CTAs per row = partial sums per row
 };
 
-// Longest chunk that still leaves kWantedCtas CTAs, but never shorter than kMinChunkQuads.
-inline RowGeometry row_geometry(long long rows, int elems, int forced_chunk_quads = 0) {
+inline RowGeometry row_geometry(long long /*rows*/, int elems, int forced_chunk_quads = 0) {
   const int quads = elems / 4;
-  int cq = kMaxChunkQuads;
-  if (forced_chunk_quads > 0) {
-    cq = forced_chunk_quads;
-  } else {
-    while (cq > kMinChunkQuads && rows * ((quads + cq - 1) / cq) < kWantedCtas) cq >>= 1;
-  }
   RowGeometry g;
-  g.chunk_quads = cq;
-  g.chunks = (quads + cq - 1) / cq;
+  g.chunk_quads = forced_chunk_quads > 0 ? forced_chunk_quads : kChunkQuads;
+  g.chunks = (quads + g.chunk_quads - 1) / g.chunk_quads;
   return g;
 }
 

@@ -219,7 +219,15 @@ int pg_step(pg_rollout* h, int32_t step, const pg_step_coef* coef, const float* 
   if (!h || !coef || !x_in || !vel || !x_out || !logp_out) return PG_EINVAL;
   if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (!aligned16(x_in) || !aligned16(vel) || !aligned16(x_out)) return PG_EINVAL;
-  if (src_rows && x_in == x_out) return PG_EINVAL;
+  if (src_rows) {
+    // a gathered step reads rows that other CTAs may already have overwritten if the output shares
+    // any byte with the input: refuse every overlap, not only x_out == x_in
+    const size_t row_bytes = (size_t)h->cfg.elems * sizeof(float);
+    const uintptr_t in_lo = (uintptr_t)x_in, out_lo = (uintptr_t)x_out;
+    const uintptr_t in_hi = in_lo + (size_t)h->cfg.n_groups * (h->k_prev > 0 ? h->k_prev : h->k_cur) * row_bytes;
+    const uintptr_t out_hi = out_lo + (size_t)h->cfg.n_groups * h->k_cur * row_bytes;
+    if (in_lo < out_hi && out_lo < in_hi) return PG_EINVAL;
+  }
   if (!(coef->noise_std >= 0.0) || !std::isfinite(coef->c_x) || !std::isfinite(coef->c_v) ||
       !std::isfinite(coef->noise_std))
     return PG_EINVAL;

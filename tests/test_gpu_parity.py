@@ -528,6 +528,9 @@ def test_out_of_sequence_calls_are_refused(B):
             B.step(h, 1, (1, 0, 0.1), x, x, src, x, lp)            # gather must not be in place
         assert e.value.code == B.EINVAL
         with pytest.raises(B.PgError) as e:
+            B.step(h, 1, (1, 0, 0.1), x, x, src, x[2:], lp)        # nor into an offset view of its input
+        assert e.value.code == B.EINVAL
+        with pytest.raises(B.PgError) as e:
             B.step(h, 1, (1, 0, -0.1), x, x, None, x, lp)          # negative noise scale
         assert e.value.code == B.EINVAL
         with pytest.raises(B.PgError) as e:
