@@ -28,11 +28,56 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) over algorithmic bytes of the step
-# kernel, from the ncu capture summarised in profiles/step_kernel_bf16_1024rows.txt (1024-row
-# launch: 2.640 GB measured, 2.684 GB algorithmic).  Set to None whenever the kernel changes
-# until the counters are taken again.
-STEP_KERNEL_TRAFFIC_RATIO = 0.984
+STEP_PROFILE = os.path.join(ROOT, "profiles", "step_kernel_bf16_256rows.txt")
+STEP_SOURCES = [os.path.join(ROOT, "paper_2512_15347_b200", "csrc", f) for f in ("pg_step.cu", "pg_common.cuh")]
+
+
+def _sources_sha256(paths=STEP_SOURCES):
+    import hashlib
+    h = hashlib.sha256()
+    for p in paths:
+        with open(p, "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def step_traffic_ratio(profile=STEP_PROFILE):
+    """DRAM bytes over algorithmic bytes of the step kernel, read from the committed ncu summary:
+    its `dram__bytes_read.sum` / `dram__bytes_write.sum` lines (first captured launch) and its
+    `algorithmic_bytes` line.  The summary also records the SHA-256 of the kernel's sources at
+    capture time; when the sources have changed since, the counters no longer describe the kernel
+    and None is returned (the bench line then carries "traffic": null)."""
+    import re
+    try:
+        text = open(profile).read()
+    except OSError:
+        return None, "no ncu summary"
+    sha = re.search(r"source_sha256:\s*([0-9a-f]{64})", text)
+    if not sha or sha.group(1) != _sources_sha256():
+        return None, "kernel sources changed since the ncu capture"
+    unit = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    vals = {}
+    for key in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+        m = re.search(re.escape(key) + r"\s+([0-9.eE+-]+)\s*(byte|Kbyte|Mbyte|Gbyte)", text)
+        if not m:
+            return None, "ncu summary lacks " + key
+        vals[key] = float(m.group(1)) * unit[m.group(2)]
+    alg = re.search(r"algorithmic_bytes:\s*([0-9]+)", text)
+    if not alg:
+        return None, "ncu summary lacks algorithmic_bytes"
+    return sum(vals.values()) / float(alg.group(1)), os.path.relpath(profile, ROOT)
+
+
+def cpu_model():
+    try:
+        for line in open("/proc/cpuinfo"):
+            if line.lower().startswith("model name"):
+                return line.split(":", 1)[1].strip()
+    except OSError:
+        pass
+    import platform
+    return platform.processor() or platform.machine()
+
 
 # the headline metric has three components: `value` is the first (latent-steps/s), the achieved HBM
 # GB/s is in `roofline` / `hbm_gbs_whole_rollout` / `prune_stage_gbs`, OVF groups/s in `ovf_microbench`
@@ -172,8 +217,8 @@ def run_reference(args):
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": mean_sec * 1e3,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
             "data": "synthetic", "config": _config(w, args),
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
-                             "sample": sample.desc + "; warm-up on 1 group"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "cpu_model": cpu_model(),
+                             "kind": "oracle", "sample": sample.desc + "; warm-up on 1 group"},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line))
@@ -386,7 +431,7 @@ def run_ours(args):
         sample = OracleSample(w, min(ORACLE_GROUPS, w.n_groups))
         sec = min(sample.run() for _ in range(2))
         cpu_base = {"value": sample.sw.traj_steps / sec, "unit": UNIT, "cores": oracle.num_threads(),
-                    "kind": "oracle", "sample": sample.desc + f"; best of 2 runs, {sec:.1f} s each"}
+                    "cpu_model": cpu_model(), "kind": "oracle", "sample": sample.desc + f"; best of 2 runs, {sec:.1f} s each"}
         del sample
         if args.workload == "large" and not args.groups and not args.no_others:
             for name, groups in OTHER_WORKLOADS:
@@ -481,6 +526,17 @@ def run_ours(args):
         ms = kinds["score"]["ms"] + kinds["prune"]["ms"]
         prune_stage_gbs = (score_bytes + kinds["prune"]["rows"] * 8) / (ms * 1e-3) / 1e9
     peak, peak_kind = _peaks()
+    traffic_ratio, traffic_note = step_traffic_ratio()
+    # the other half of the target: the prune stage (latent scoring + OVF selection) as one unit
+    also = []
+    if score_gbs is not None:
+        also.append({"kernel": "score_kernel (latent score, read-only)", "bound": "hbm", "achieved": score_gbs,
+                     "peak": peak, "unit": "GB/s", "frac": score_gbs / peak, "bytes_per_element": 4 + vel_bytes})
+    if prune_stage_gbs is not None:
+        also.append({"kernel": "score + ovf (prune stage: scoring pass and selection launch together)",
+                     "bound": "hbm", "achieved": prune_stage_gbs, "peak": peak, "unit": "GB/s",
+                     "frac": prune_stage_gbs / peak,
+                     "bytes": "6 B per scored element + 8 B per score / kept index"})
 
     # OVF selection microbenchmark (4096 groups x 256 scores -> 32) on rank 0
     ovf = None
@@ -627,10 +683,12 @@ def run_ours(args):
                              "frac": step_gbs / peak, "peak_kind": peak_kind,
                              "frac_of_8TBs_nominal": step_gbs / 8000.0,
                              "bytes_per_launch": step_bytes / kinds["step"]["launches"],
-                             "traffic": (None if STEP_KERNEL_TRAFFIC_RATIO is None else
-                                         STEP_KERNEL_TRAFFIC_RATIO * step_bytes / kinds["step"]["launches"]),
-                             "traffic_source": "ncu capture of the 1024-row launch, scaled by rows "
-                                               "(traffic is proportional to rows x elements)",
+                             "traffic": (None if traffic_ratio is None else
+                                         traffic_ratio * step_bytes / kinds["step"]["launches"]),
+                             "traffic_source": traffic_note if traffic_ratio is None else
+                                               f"{traffic_note}: DRAM / algorithmic bytes = {traffic_ratio:.4f} on the captured "
+                                               "256-row launch, scaled by rows (every element is read and written once)",
+                             "also": also,
                              "bytes_per_element_step": 8 + vel_bytes},
                 "kernels": {k: {"ms_per_rollout": v["ms"] / args.steps, "launches_per_rollout":
                                 v["launches"] // args.steps} for k, v in kinds.items()},
