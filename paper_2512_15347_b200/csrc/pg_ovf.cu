@@ -1,11 +1,11 @@
 // Optimal Variance Filtering (Eq. "ovf"), survivor index compaction, group-relative advantages
 // (Eq. "advK"), clustering diagnostics and the uniform-subsampling baseline.
 //
-// Selection: one warp per group; the scores become order-preserving 32-bit keys, are sorted in
+// Selection: one warp (or half a warp) per group; the scores become order-preserving 32-bit keys, are sorted in
 // registers, the running sums from both ends give the k+1 candidate variances "j lowest + (k-j)
 // highest" in fp64 with explicitly rounded operations, membership follows from the keys at the
 // two cuts (from ranks in the total order (score, slot) when keys tie there), and the kept slots
-// are written in ascending slot order through a popcount prefix sum.
+// are written in ascending slot order through ballots and popcounts.
 #include "pg_common.cuh"
 #include <float.h>
 
@@ -46,14 +46,22 @@ __device__ __forceinline__ double arithmetic_value(float s) {
 
 // ---------------------------------------------------------------- selection kernel
 //
-// One warp per group, E = 1, 2, 4, 8, 16 or 32 scores per lane (n <= 32 * E <= 1024); the warps
-// of a CTA (four, or one for the widest groups) only meet once, for the staging of their rows.
+// A group of n scores is handled by the W lanes of a warp (W = 32 in every instantiation the
+// launcher uses), E scores per lane, n <= W * E <= 1024.  The kernel is written for W = 16 as
+// well - two groups per warp, one per half, so that the phases which use few lanes per group
+// (serial running sums, candidate argmax, prefix counts, advantage statistics) serve two groups
+// at once - but on the 4096 x 256 -> 32 shape that variant was no faster (each lane then sorts
+// twice as many keys and half as many warps are left to hide latencies), so it is not dispatched.
+// The warps of a CTA only meet once, for the staging of their rows.
 //  0. The CTA's score rows are staged in shared memory by one bulk asynchronous copy
 //     (cp.async.bulk, completion on an mbarrier, bounded wait) when source and size are
-//     16-byte aligned, else read with ordinary loads.
+//     16-byte aligned, else read with ordinary loads.  Lane l takes slots l, l + W, l + 2W, ...
+//     (consecutive lanes read consecutive words: no bank conflicts, coalesced global loads).
 //  1. The 32-bit order keys alone are sorted with a bitonic network held in registers (one
 //     integer min and one max per compare-exchange; shuffles for distances of E and more).
-//     Slots >= n hold an all-ones key and sort to the end.
+//     Slots >= n hold an all-ones key and sort to the end.  Sorted position q sits in register
+//     q % E of lane q / E and is kept in shared memory at word (q % E) * W + q / E, again so that
+//     consecutive lanes store consecutive words.
 //  2. Running sums from both ends: the centred values and their squares are formed by all lanes
 //     in parallel, then lanes 0..3 accumulate one sequence each serially, in order, in fp64 with
 //     explicitly rounded operations - the same operations in the same order as a plain serial loop.
@@ -61,36 +69,55 @@ __device__ __forceinline__ double arithmetic_value(float s) {
 //  4. Membership: by comparison with the two keys at the cuts of the order; only when a key just
 //     inside a cut equals the one just outside it (rare for real scores) is the rank of every
 //     element in the total order (score, slot) worked out, by a binary search in the sorted keys
-//     plus a direct count of equal keys in lower slots.  Every lane holds its scores in slot
-//     order, so a popcount prefix over lanes gives ascending slot order.
+//     plus a direct count of equal keys in lower slots.  Ascending slot order of the kept slots
+//     follows from one ballot per register index (slots r * W + lane are ascending in r, then lane).
 //  5. Kept scores go through shared memory so that their stores, the advantage statistics and
 //     the single division are spread over the lanes.
-// warps (= groups) per CTA: four while the per-warp shared memory allows it, one for wide groups
-template <int E> struct OvfWarps { static constexpr int value = (E <= 8) ? 4 : 1; };
+constexpr int kOvfMaxWarps = 4;                 // warps per CTA, fewer when the groups' shared memory is large
+constexpr size_t kOvfSmemBudget = 47 * 1024;    // dynamic shared memory a CTA may use without opting in
 
 __device__ __forceinline__ float key_to_score(uint32_t key) {
   const uint32_t b = (key & 0x80000000u) ? (key ^ 0x80000000u) : ~key;
   return __uint_as_float(b);      // all-ones key -> 0x7FFFFFFF, a NaN, as it went in
 }
 
-template <int E>
-__global__ void __launch_bounds__(OvfWarps<E>::value * 32)
+template <int W>
+__device__ __forceinline__ double lanes_sum(double v) {      // sum over the W lanes of a group
+#pragma unroll
+  for (int o = W / 2; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  return v;
+}
+
+// bytes of shared memory per group: four running-sum arrays of k + 1 doubles, sorted keys and
+// slot-order keys of W * E words each (the staged row comes on top: W * E floats)
+__host__ __device__ inline size_t ovf_group_bytes(int k, int N) {
+  return (size_t)(k + 1) * 4 * sizeof(double) + (size_t)N * 2 * sizeof(uint32_t);
+}
+
+template <int E, int W>
+__global__ void __launch_bounds__(kOvfMaxWarps * 32)
 ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
-  constexpr int N = 32 * E;
-  constexpr int kOvfWarpsPerCta = OvfWarps<E>::value;
+  constexpr int N = W * E;
+  constexpr int kPerWarp = 32 / W;                       // groups per warp
+  constexpr unsigned int kFull = 0xFFFFFFFFu;
   extern __shared__ __align__(16) unsigned char smem[];
   __shared__ __align__(8) unsigned long long stage_bar;
   const int n = p.n, k = p.k;
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int g0 = blockIdx.x * kOvfWarpsPerCta;
-  const int g = g0 + warp;
+  const int groups_per_cta = (blockDim.x >> 5) * kPerWarp;
+  const int warp = threadIdx.x >> 5, wlane = threadIdx.x & 31;
+  const int lane = wlane & (W - 1), sub = wlane / W;     // lane within the group, group within the warp
+  const int slot = warp * kPerWarp + sub;                // group within the CTA
+  const int g0 = blockIdx.x * groups_per_cta;
+  const int g = g0 + slot;
+  const bool active = g < n_groups;                      // a warp's second half may have no group
 
   // 0. stage the score rows of this CTA's groups (contiguous in memory) in shared memory with
   //    one bulk asynchronous copy, completion signalled on an mbarrier.  Needs a 16-byte
   //    aligned source and size; otherwise the rows are read with ordinary loads.  The wait is
-  //    bounded: if the copy has not landed in time, status bit 1 is set and the CTA gives up.
-  float* stage = reinterpret_cast<float*>(smem);                 // [kOvfWarpsPerCta * n]
-  const int groups_here = min(kOvfWarpsPerCta, n_groups - g0);
+  //    bounded: if the copy has not landed in time, status bit 1 is set, the wait is repeated
+  //    once, and if any thread still has not seen the copy land the whole CTA gives up together.
+  float* stage = reinterpret_cast<float*>(smem);                 // [groups_per_cta * N]
+  const int groups_here = min(groups_per_cta, n_groups - g0);
   const unsigned int stage_bytes = (unsigned int)groups_here * (unsigned int)n * 4u;
   const bool bulk = p.bulk_ok && (stage_bytes & 15u) == 0 && ((((size_t)g0 * n * 4) & 15) == 0);
   if (bulk) {                                                    // uniform over the CTA
@@ -115,27 +142,33 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
       done = mbarrier_wait_bounded(bar, 0u, kBulkWaitLimit);
       if (!done && round == 0 && threadIdx.x == 0 && p.status) atomicOr(p.status, 2);
     }
-    if (!done) return;        // waited twice without success: leave, the host reads the status
+    // one verdict for the CTA: threads whose last attempt succeeded must not run ahead into the
+    // warp-wide shuffles while others of their warp leave
+    if (!__syncthreads_and(done ? 1 : 0)) {
+      if (threadIdx.x == 0 && p.status) atomicOr(p.status, 2);
+      return;
+    }
   }
-  if (g >= n_groups) return;
-  const size_t per_warp = (size_t)(k + 1) * 4 * sizeof(double) + (size_t)N * 2 * sizeof(uint32_t);
-  unsigned char* base = smem + (size_t)kOvfWarpsPerCta * N * sizeof(float) + (size_t)warp * per_warp;
+  if (g0 + warp * kPerWarp >= n_groups) return;                  // the whole warp has no group
+  const size_t per_group = ovf_group_bytes(k, N);
+  unsigned char* base = smem + (size_t)groups_per_cta * N * sizeof(float) + (size_t)slot * per_group;
   double* L1 = reinterpret_cast<double*>(base);
   double* L2 = L1 + (k + 1);
   double* H1 = L2 + (k + 1);
   double* H2 = H1 + (k + 1);
-  uint32_t* skey = reinterpret_cast<uint32_t*>(H2 + (k + 1));   // [N] sorted keys
+  uint32_t* skey = reinterpret_cast<uint32_t*>(H2 + (k + 1));   // [N] sorted keys, position q at (q % E) * W + q / E
   uint32_t* okey = skey + N;                                    // [N] keys in slot order
+  auto sorted_key = [&](int q) -> uint32_t { return skey[(q & (E - 1)) * W + (q / E)]; };
 
-  const float* sc = p.scores + (size_t)g * n;
+  const float* sc = p.scores + (size_t)(active ? g : 0) * n;
   float orig[E];
   uint32_t mine[E], key[E];
   bool bad = false;
 #pragma unroll
   for (int r = 0; r < E; ++r) {
-    const int i = lane * E + r;
-    if (i < n) {
-      orig[r] = bulk ? stage[warp * n + i] : sc[i];
+    const int i = r * W + lane;                                  // slot within the group
+    if (active && i < n) {
+      orig[r] = bulk ? stage[slot * n + i] : sc[i];
       bad |= !(fabsf(orig[r]) <= FLT_MAX);
       mine[r] = order_key(orig[r]);
     } else {
@@ -146,8 +179,9 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
   }
   if (bad && p.status) atomicOr(p.status, 1);
 
-  // 1. bitonic sort, ascending over index lane * E + r; every compare-exchange points the same
-  //    way: a merge first pairs i with its mirror i ^ (size - 1), then halves the distance.
+  // 1. bitonic sort, ascending over position lane * E + r; every compare-exchange points the same
+  //    way: a merge first pairs a position with its mirror q ^ (size - 1), then halves the distance.
+  //    (Which slot starts in which register does not matter to a sort.)
 #pragma unroll
   for (int size = 2; size <= N; size <<= 1) {
     if (size <= E) {
@@ -165,7 +199,7 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
       const bool lower = (lane & (size / E / 2)) == 0;
       uint32_t other[E];
 #pragma unroll
-      for (int r = 0; r < E; ++r) other[r] = __shfl_xor_sync(0xFFFFFFFFu, key[r ^ (E - 1)], lane_mask);
+      for (int r = 0; r < E; ++r) other[r] = __shfl_xor_sync(kFull, key[r ^ (E - 1)], lane_mask);
 #pragma unroll
       for (int r = 0; r < E; ++r) key[r] = lower ? min(key[r], other[r]) : max(key[r], other[r]);
     }
@@ -185,21 +219,21 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
         const bool lower = (lane & lane_mask) == 0;
 #pragma unroll
         for (int r = 0; r < E; ++r) {
-          const uint32_t other = __shfl_xor_sync(0xFFFFFFFFu, key[r], lane_mask);
+          const uint32_t other = __shfl_xor_sync(kFull, key[r], lane_mask);
           key[r] = lower ? min(key[r], other) : max(key[r], other);
         }
       }
     }
   }
 #pragma unroll
-  for (int r = 0; r < E; ++r) skey[lane * E + r] = key[r];
+  for (int r = 0; r < E; ++r) skey[r * W + lane] = key[r];
   __syncwarp();
 
-  // 3. centred values and squares in parallel, then the serial running sums
-  const double pivot = arithmetic_value(key_to_score(skey[n / 2]));
-  for (int j = lane; j < k; j += 32) {
-    const double cl = __dsub_rn(arithmetic_value(key_to_score(skey[j])), pivot);
-    const double ch = __dsub_rn(arithmetic_value(key_to_score(skey[n - 1 - j])), pivot);
+  // 2. centred values and squares in parallel, then the serial running sums
+  const double pivot = arithmetic_value(key_to_score(sorted_key(n / 2)));
+  for (int j = lane; j < k; j += W) {
+    const double cl = __dsub_rn(arithmetic_value(key_to_score(sorted_key(j))), pivot);
+    const double ch = __dsub_rn(arithmetic_value(key_to_score(sorted_key(n - 1 - j))), pivot);
     L1[j + 1] = cl;
     L2[j + 1] = __dmul_rn(cl, cl);
     H1[j + 1] = ch;
@@ -218,57 +252,59 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
   }
   __syncwarp();
 
-  // 4. candidates
+  // 3. candidates
   double best_m = -1.0;
   int best_j = -1;
-  for (int j = lane; j <= k; j += 32) {
+  for (int j = lane; j <= k; j += W) {
     const double S = __dadd_rn(L1[j], H1[k - j]);
     const double Q = __dadd_rn(L2[j], H2[k - j]);
     const double M = __dsub_rn(__dmul_rn((double)k, Q), __dmul_rn(S, S));
     if (best_j < 0 || M >= best_m) { best_m = M; best_j = j; }
   }
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const double om = __shfl_xor_sync(0xFFFFFFFFu, best_m, o);
-    const int oj = __shfl_xor_sync(0xFFFFFFFFu, best_j, o);
+  for (int o = W / 2; o > 0; o >>= 1) {
+    const double om = __shfl_xor_sync(kFull, best_m, o);
+    const int oj = __shfl_xor_sync(kFull, best_j, o);
     if (oj >= 0 && (best_j < 0 || om > best_m || (om == best_m && oj > best_j))) {
       best_m = om; best_j = oj;
     }
   }
   const int jstar = best_j;
   const int high_from = n - (k - jstar);
-  if (lane == 0 && p.sel_var) p.sel_var[g] = (float)(best_m / ((double)k * (double)k));
+  if (lane == 0 && active && p.sel_var) p.sel_var[g] = (float)(best_m / ((double)k * (double)k));
 
-  // 5. membership.  With distinct keys at both cuts of the order an element is kept exactly when
+  // 4. membership.  With distinct keys at both cuts of the order an element is kept exactly when
   //    its key is at most the j*-th lowest or at least the (k - j*)-th highest key.  Only when the
   //    key just inside a cut equals the key just outside it does the slot decide: then every
   //    element finds its rank in the total order (score, slot) by a binary search for its key in
   //    the sorted list, advanced by the number of equal keys in lower slots.
   const int n_high = k - jstar;
-  const uint32_t lowkey = jstar > 0 ? skey[jstar - 1] : 0u;
-  const uint32_t highkey = n_high > 0 ? skey[high_from] : 0xFFFFFFFFu;
-  const bool cut_tie = (jstar > 0 && jstar < n && skey[jstar] == lowkey) ||
-                       (n_high > 0 && high_from > 0 && skey[high_from - 1] == highkey);
+  const uint32_t lowkey = jstar > 0 ? sorted_key(jstar - 1) : 0u;
+  const uint32_t highkey = n_high > 0 ? sorted_key(high_from) : 0xFFFFFFFFu;
+  const bool cut_tie = (jstar > 0 && jstar < n && sorted_key(jstar) == lowkey) ||
+                       (n_high > 0 && high_from > 0 && sorted_key(high_from - 1) == highkey);
+  if (__any_sync(kFull, cut_tie)) {                 // uniform over the warp: both groups publish their keys
+#pragma unroll
+    for (int r = 0; r < E; ++r) okey[r * W + lane] = mine[r];
+    __syncwarp();
+  }
   unsigned int bits = 0u;
-  if (!cut_tie) {                                   // uniform over the warp
+  if (!cut_tie) {                                   // uniform over the group; no warp-wide operation inside
 #pragma unroll
     for (int r = 0; r < E; ++r) {
       const bool in_low = jstar > 0 && mine[r] <= lowkey;
       const bool in_high = n_high > 0 && mine[r] >= highkey;
-      if (lane * E + r < n && (in_low || in_high)) bits |= 1u << r;
+      if (r * W + lane < n && (in_low || in_high)) bits |= 1u << r;
     }
   } else {
 #pragma unroll
-    for (int r = 0; r < E; ++r) okey[lane * E + r] = mine[r];
-    __syncwarp();
-#pragma unroll
     for (int r = 0; r < E; ++r) {
-      const int i = lane * E + r;
+      const int i = r * W + lane;
       int rank = 0;
 #pragma unroll
       for (int step = N / 2; step > 0; step >>= 1)
-        if (skey[rank + step - 1] < mine[r]) rank += step;    // first position whose key is >= mine
-      if (i < n && rank + 1 < N && skey[rank + 1] == mine[r]) {  // equal keys exist
+        if (sorted_key(rank + step - 1) < mine[r]) rank += step;    // first position whose key is >= mine
+      if (i < n && rank + 1 < N && sorted_key(rank + 1) == mine[r]) {  // equal keys exist
         int lower_slots = 0;
         for (int j = 0; j < i; ++j) lower_slots += (okey[j] == mine[r]) ? 1 : 0;
         rank += lower_slots;
@@ -276,60 +312,61 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
       if (i < n && (rank < jstar || rank >= high_from)) bits |= 1u << r;
     }
   }
-  const int cnt = __popc(bits);
-  int incl = cnt;
-#pragma unroll
-  for (int o = 1; o < 32; o <<= 1) {
-    const int t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-    if (lane >= o) incl += t;
-  }
-  const int first = lane * E;
+
+  // 5. output in ascending slot order: slots r * W + lane ascend with r first, then with the lane
   const bool want_scores = p.kept_scores || p.adv;
   float* kept_s = reinterpret_cast<float*>(L1);     // [k], reuses the running sums' space
   __syncwarp();                                     // every lane is done with the running sums
-  int pos = incl - cnt;
+  constexpr unsigned int kGroupMask = (W == 32) ? 0xFFFFFFFFu : ((1u << (W & 31)) - 1u);
+  int before = 0;                                   // kept slots of this group below the current r
 #pragma unroll
   for (int r = 0; r < E; ++r) {
-    if (bits & (1u << r)) {
-      const int i = first + r;
+    const bool kept = (bits >> r) & 1u;
+    const unsigned int group_votes = (__ballot_sync(kFull, kept) >> (sub * W)) & kGroupMask;
+    if (kept && active) {
+      const int i = r * W + lane;
+      const int pos = before + __popc(group_votes & ((1u << lane) - 1u));
       const size_t o = (size_t)g * k + pos;
       p.keep_idx[o] = i;
       if (p.src_rows) p.src_rows[o] = g * n + i;
       if (p.traj_out) p.traj_out[o] = p.traj_in[(size_t)g * n + i];
       if (want_scores) kept_s[pos] = orig[r];
-      ++pos;
     }
+    before += __popc(group_votes);
   }
   if (want_scores) {
     // kept scores in slot order, now spread over the lanes: coalesced stores, one division
     __syncwarp();
     double sum_kept = 0.0;
-    for (int j = lane; j < k; j += 32) {
+    for (int j = lane; j < k; j += W) {
       const float v = kept_s[j];
-      if (p.kept_scores) p.kept_scores[(size_t)g * k + j] = v;
+      if (p.kept_scores && active) p.kept_scores[(size_t)g * k + j] = v;
       sum_kept += (double)v;
     }
     if (p.adv) {
-      const double mu = warp_sum(sum_kept) / (double)k;
+      const double mu = lanes_sum<W>(sum_kept) / (double)k;
       double sq = 0.0;
-      for (int j = lane; j < k; j += 32) {
+      for (int j = lane; j < k; j += W) {
         const double dlt = (double)kept_s[j] - mu;
         sq += dlt * dlt;
       }
-      const double inv = 1.0 / (sqrt(warp_sum(sq) / (double)k) + (double)p.adv_eps);
-      for (int j = lane; j < k; j += 32)
-        p.adv[(size_t)g * k + j] = (float)(((double)kept_s[j] - mu) * inv);
+      const double inv = 1.0 / (sqrt(lanes_sum<W>(sq) / (double)k) + (double)p.adv_eps);
+      if (active)
+        for (int j = lane; j < k; j += W)
+          p.adv[(size_t)g * k + j] = (float)(((double)kept_s[j] - mu) * inv);
     }
   }
 }
 
-template <int E>
+template <int E, int W>
 static void launch_ovf_warp(const OvfParams& p, int n_groups, cudaStream_t stream) {
-  const size_t per_warp = (size_t)(p.k + 1) * 4 * sizeof(double) + (size_t)(32 * E) * 2 * sizeof(uint32_t);
-  constexpr int kOvfWarpsPerCta = OvfWarps<E>::value;
-  const size_t stage = (size_t)kOvfWarpsPerCta * 32 * E * sizeof(float);
-  const int ctas = (n_groups + kOvfWarpsPerCta - 1) / kOvfWarpsPerCta;
-  ovf_warp_kernel<E><<<ctas, kOvfWarpsPerCta * 32, stage + per_warp * kOvfWarpsPerCta, stream>>>(p, n_groups);
+  constexpr int N = W * E, kPerWarp = 32 / W;
+  const size_t per_group = ovf_group_bytes(p.k, N) + (size_t)N * sizeof(float);   // + the staged row
+  int warps = kOvfMaxWarps;
+  while (warps > 1 && (size_t)warps * kPerWarp * per_group > kOvfSmemBudget) warps >>= 1;
+  const int groups_per_cta = warps * kPerWarp;
+  const int ctas = (n_groups + groups_per_cta - 1) / groups_per_cta;
+  ovf_warp_kernel<E, W><<<ctas, warps * 32, (size_t)groups_per_cta * per_group, stream>>>(p, n_groups);
 }
 
 int launch_ovf(int n_groups, int n, int k, const float* scores, int32_t* keep_idx,
@@ -350,12 +387,12 @@ int launch_ovf(int n_groups, int n, int k, const float* scores, int32_t* keep_id
   p.k = k;
   p.adv_eps = adv_eps;
   p.bulk_ok = (((uintptr_t)scores) & 15) == 0;
-  if (n <= 32)       launch_ovf_warp<1>(p, n_groups, stream);
-  else if (n <= 64)  launch_ovf_warp<2>(p, n_groups, stream);
-  else if (n <= 128) launch_ovf_warp<4>(p, n_groups, stream);
-  else if (n <= 256) launch_ovf_warp<8>(p, n_groups, stream);
-  else if (n <= 512) launch_ovf_warp<16>(p, n_groups, stream);
-  else launch_ovf_warp<32>(p, n_groups, stream);
+  if (n <= 32)       launch_ovf_warp<1, 32>(p, n_groups, stream);
+  else if (n <= 64)  launch_ovf_warp<2, 32>(p, n_groups, stream);
+  else if (n <= 128) launch_ovf_warp<4, 32>(p, n_groups, stream);
+  else if (n <= 256) launch_ovf_warp<8, 32>(p, n_groups, stream);
+  else if (n <= 512) launch_ovf_warp<16, 32>(p, n_groups, stream);
+  else               launch_ovf_warp<32, 32>(p, n_groups, stream);
   PG_LAUNCH_CHECK();
   return PG_OK;
 }
@@ -512,6 +549,7 @@ __global__ void __launch_bounds__(32) wait_selftest_kernel(int32_t* status) {
     done = mbarrier_wait_bounded(bar, 0u, kBulkWaitLimit);
     if (!done && round == 0 && threadIdx.x == 0 && status) atomicOr(status, 2);
   }
+  if (!__syncthreads_and(done ? 1 : 0)) return;      // the same CTA-wide verdict as in the selection kernel
 }
 
 int launch_wait_selftest(int32_t* status, cudaStream_t stream) {
