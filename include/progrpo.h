@@ -265,7 +265,9 @@ int pg_policy_logprob(pg_rollout *h, const pg_step_coef *coef, const float *x, c
  * (nullable), ratio (nullable, out), dlogp (out) are [n_steps, n_active] fp32; adv [n_active].
  * dlogp = d objective / d logp_new: A r / (n_steps n_active) where the unclipped branch is
  * active, else 0.  The matching derivative with respect to kl is the constant
- * -beta / (n_steps n_active).  Evaluated in fp64 from the fp32 inputs; one small launch.
+ * -beta / (n_steps n_active).  Evaluated in fp64 from the fp32 inputs; one launch of as many
+ * CTAs as the entries need, their partial sums combined in a fixed order (the same bits on every
+ * run); uses the handle's scratch, so calls on one handle must be ordered like all others.
  */
 int pg_policy_objective(pg_rollout *h, int32_t n_steps, const float *logp_new, const float *logp_old,
                         const float *kl, const float *adv, float clip_eps, float beta, float *ratio,
@@ -323,6 +325,22 @@ int pg_rollout_host(const pg_config *cfg, const pg_step_coef *step_coef,
                     const void *const *vel_steps, const float *const *stage_scores,
                     const float *final_rewards, float *x_final, float *logp, int32_t *keep_idx,
                     float *adv, int32_t *traj_id, void *workspace, size_t workspace_bytes);
+
+/*
+ * The same whole rollout from HOST buffers on an existing handle (Section 5.1 + 5.2 end to end):
+ * pg_rollout_host creates and destroys a handle - six device allocations and a device
+ * synchronisation - on every call, which dominates the call for small latents; a caller that
+ * rolls out the same schedule repeatedly creates the handle once and calls this instead.  The
+ * handle is rewound first; its two streams and four events are created on the first call and
+ * released by pg_rollout_destroy, so later calls allocate nothing.  Arguments, layout of the
+ * outputs and the workspace are those of pg_rollout_host (schedule = the handle's); synchronises
+ * before returning.
+ */
+int pg_rollout_host_on(pg_rollout *h, const pg_step_coef *step_coef,
+                       const pg_preview_coef *preview_coef, const float *x0,
+                       const void *const *vel_steps, const float *const *stage_scores,
+                       const float *final_rewards, float *x_final, float *logp, int32_t *keep_idx,
+                       float *adv, int32_t *traj_id, void *workspace, size_t workspace_bytes);
 
 /*
  * Latent score without any allocation (no counterpart in the paper: this is a packaging

@@ -90,6 +90,8 @@ def lib() -> ctypes.CDLL:
     L.pg_rollout_host.argtypes = [ctypes.POINTER(Config), ctypes.POINTER(StepCoef),
                                   ctypes.POINTER(PreviewCoef), vp, ctypes.POINTER(vp),
                                   ctypes.POINTER(vp), vp, vp, vp, vp, vp, vp, vp, sz]
+    L.pg_rollout_host_on.argtypes = [vp, ctypes.POINTER(StepCoef), ctypes.POINTER(PreviewCoef), vp,
+                                     ctypes.POINTER(vp), ctypes.POINTER(vp), vp, vp, vp, vp, vp, vp, vp, sz]
     L.pg_score_static.argtypes = [i32, i32, i32, ctypes.POINTER(PreviewCoef), vp, vp, vp, vp]
     L.pg_rollout_run_workspace_bytes.argtypes = [ctypes.POINTER(Config)]
     L.pg_rollout_run_workspace_bytes.restype = sz
@@ -111,7 +113,7 @@ def lib() -> ctypes.CDLL:
                  "pg_step", "pg_score", "pg_prune_ovf", "pg_compact", "pg_advantages",
                  "pg_ovf_select_batched", "pg_rollout_host", "pg_rollout_traj_ids",
                  "pg_philox_raw", "pg_normal_rows", "pg_score_static", "pg_policy_logprob",
-                 "pg_policy_objective", "pg_policy_backward", "pg_prune_uniform", "pg_group_stats", "pg_preview", "pg_rollout_run", "pg_rollout_restore", "pg_score_preview"):
+                 "pg_policy_objective", "pg_policy_backward", "pg_prune_uniform", "pg_group_stats", "pg_preview", "pg_rollout_run", "pg_rollout_restore", "pg_score_preview", "pg_rollout_host_on"):
         getattr(L, name).restype = ctypes.c_int
     _lib = L
     return L
@@ -324,6 +326,31 @@ def rollout_host(cfg: Config, step_coefs, preview_coefs, x0, vel_steps, stage_sc
                                _p(workspace), workspace.numel() * workspace.element_size())
     if rc not in (OK, ENONFINITE):
         raise PgError(rc, "pg_rollout_host")
+    return rc
+
+
+class HostArgs:
+    """Marshalled arguments of pg_rollout_host_on, built once and reused call after call."""
+
+    def __init__(self, step_coefs, preview_coefs, vel_steps, stage_scores=None):
+        self.sc = (StepCoef * len(step_coefs))(*[StepCoef(*c) for c in step_coefs])
+        self.pc = (PreviewCoef * max(len(preview_coefs), 1))(*[PreviewCoef(*c) for c in preview_coefs])
+        self.vs = (ctypes.c_void_p * len(vel_steps))(*[_p(v) for v in vel_steps])
+        self.ss = None
+        if stage_scores is not None:
+            self.ss = (ctypes.c_void_p * max(len(stage_scores), 1))(*[_p(s) for s in stage_scores])
+        self.keep = (vel_steps, stage_scores)      # the host tensors must outlive the calls
+
+
+def rollout_host_on(h: int, args: "HostArgs", x0, final_rewards, x_final, logp, keep_idx, adv, traj_id,
+                    workspace) -> int:
+    """Whole rollout from host tensors on an existing handle (see pg_rollout_host_on): no
+    allocation per call.  Returns the status code, raising for anything but OK / ENONFINITE."""
+    rc = lib().pg_rollout_host_on(h, args.sc, args.pc, _p(x0), args.vs, args.ss, _p(final_rewards),
+                                  _p(x_final), _p(logp), _p(keep_idx), _p(adv), _p(traj_id),
+                                  _p(workspace), workspace.numel() * workspace.element_size())
+    if rc not in (OK, ENONFINITE):
+        raise PgError(rc, "pg_rollout_host_on")
     return rc
 
 

@@ -282,7 +282,8 @@ int launch_policy_logprob(int n_rows, int elems, int vel_dtype, const float* x, 
 
 int launch_policy_objective(int n_steps, int n_rows, const float* logp_new, const float* logp_old,
                             const float* kl, const float* adv, float clip_eps, float beta,
-                            float* ratio, float* dlogp, float* objective, cudaStream_t stream);
+                            float* ratio, float* dlogp, float* objective, double* cta_part,
+                            unsigned int* ticket, cudaStream_t stream);
 
 int launch_policy_backward(int n_rows, int elems, int vel_dtype, const float* x, const float* x_next,
                            const void* vel, const void* vel_ref, double c_x, double c_v,

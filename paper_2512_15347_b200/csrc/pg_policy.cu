@@ -140,19 +140,27 @@ int launch_policy_logprob(int n_rows, int elems, int vel_dtype, const float* x, 
 // ---------------------------------------------------------------- clipped surrogate objective
 
 constexpr int kObjThreads = 1024;
+constexpr int kObjMinEntries = 8 * kObjThreads;      // entries per CTA: at least eight per thread
 
-// One CTA: ratios, clipped surrogate, dJ/dlogp for all (step, trajectory) pairs and the mean
-// objective, summed per thread in index order and combined in a fixed tree (fp64).
+// Ratios, clipped surrogate, dJ/dlogp for all (step, trajectory) pairs and the mean objective.
+// CTA b handles the entries [b * per_cta, (b + 1) * per_cta): every thread sums its entries in
+// index order, the CTA combines them in a fixed tree (fp64) and stores its partial sum in slot b;
+// the CTA that draws the last ticket adds the slots in slot order.  The split depends only on
+// the number of entries, so the objective is the same bits on every run.
 __global__ void __launch_bounds__(kObjThreads)
-policy_objective_kernel(int n_steps, int n_rows, const float* logp_new, const float* logp_old,
-                        const float* kl, const float* adv, float clip_eps, float beta,
-                        float* ratio, float* dlogp, float* objective) {
+policy_objective_kernel(int n_steps, int n_rows, long long per_cta, const float* logp_new,
+                        const float* logp_old, const float* kl, const float* adv, float clip_eps,
+                        float beta, float* ratio, float* dlogp, float* objective, double* cta_part,
+                        unsigned int* ticket) {
   __shared__ double part[kObjThreads / 32];
+  __shared__ int is_last;
   const long long total = (long long)n_steps * n_rows;
   const double inv = 1.0 / (double)total;
   const double lo = 1.0 - (double)clip_eps, hi = 1.0 + (double)clip_eps;
+  const long long begin = (long long)blockIdx.x * per_cta;
+  const long long end = begin + per_cta < total ? begin + per_cta : total;
   double acc = 0.0;
-  for (long long j = threadIdx.x; j < total; j += kObjThreads) {
+  for (long long j = begin + threadIdx.x; j < end; j += kObjThreads) {
     const int i = (int)(j % n_rows);
     const double r = exp((double)logp_new[j] - (double)logp_old[j]);
     const double rc = r < lo ? lo : (r > hi ? hi : r);
@@ -165,18 +173,51 @@ policy_objective_kernel(int n_steps, int n_rows, const float* logp_new, const fl
   acc = warp_sum(acc);
   if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = acc;
   __syncthreads();
-  if (threadIdx.x < 32) {
-    double v = part[threadIdx.x];
-    v = warp_sum(v);
+  double v = 0.0;
+  if (threadIdx.x < 32) v = warp_sum(part[threadIdx.x]);
+  if (gridDim.x == 1) {
     if (threadIdx.x == 0) objective[0] = (float)(v * inv);
+    return;
+  }
+  if (threadIdx.x == 0) {
+    cta_part[blockIdx.x] = v;
+    __threadfence();
+    is_last = atomicAdd(ticket, 1u) == gridDim.x - 1u;
+  }
+  __syncthreads();
+  if (!is_last) return;
+  __threadfence();
+  // slots in slot order: thread t takes slot t (at most kObjThreads slots), then the same tree
+  double s = threadIdx.x < gridDim.x ? __ldcg(cta_part + threadIdx.x) : 0.0;
+  s = warp_sum(s);
+  __syncthreads();                       // part[] is reused
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    const double w = warp_sum(part[threadIdx.x]);
+    if (threadIdx.x == 0) {
+      objective[0] = (float)(w * inv);
+      *ticket = 0u;                      // ready for the next launch
+    }
   }
 }
 
 int launch_policy_objective(int n_steps, int n_rows, const float* logp_new, const float* logp_old,
                             const float* kl, const float* adv, float clip_eps, float beta,
-                            float* ratio, float* dlogp, float* objective, cudaStream_t stream) {
-  policy_objective_kernel<<<1, kObjThreads, 0, stream>>>(n_steps, n_rows, logp_new, logp_old, kl, adv,
-                                                         clip_eps, beta, ratio, dlogp, objective);
+                            float* ratio, float* dlogp, float* objective, double* cta_part,
+                            unsigned int* ticket, cudaStream_t stream) {
+  const long long total = (long long)n_steps * n_rows;
+  if (total == 0) return PG_OK;
+  // entries per CTA: kObjMinEntries, or more (a multiple of the CTA size) so that kObjThreads slots suffice
+  long long per_cta = kObjMinEntries;
+  if ((total + per_cta - 1) / per_cta > kObjThreads) {
+    per_cta = (total + kObjThreads - 1) / kObjThreads;
+    per_cta = (per_cta + kObjThreads - 1) / kObjThreads * kObjThreads;
+  }
+  const unsigned int ctas = (unsigned int)((total + per_cta - 1) / per_cta);
+  policy_objective_kernel<<<ctas, kObjThreads, 0, stream>>>(n_steps, n_rows, per_cta, logp_new, logp_old, kl,
+                                                            adv, clip_eps, beta, ratio, dlogp, objective,
+                                                            cta_part, ticket);
   PG_LAUNCH_CHECK();
   return PG_OK;
 }

@@ -39,6 +39,11 @@ struct pg_rollout {
   float* d_partials = nullptr;
   unsigned int* d_tickets = nullptr;
   int32_t* d_status = nullptr;
+  double* d_obj_part = nullptr;        // [1024] per-CTA partial sums of the objective kernel
+  unsigned int* d_obj_ticket = nullptr; // its arrival counter, zero between launches
+  // streams and events of the host-buffer driver, created on its first use with this handle
+  cudaStream_t host_compute = nullptr, host_copy = nullptr;
+  cudaEvent_t v_ready[2] = {nullptr, nullptr}, v_free[2] = {nullptr, nullptr};
   long long* d_step_off = nullptr;   // [T + 1] offsets of the steps in a packed per-step row array
   long long total_step_rows = 0;
 };
@@ -114,6 +119,9 @@ int pg_rollout_init(const pg_config* cfg, pg_rollout** out) {
   if (e == cudaSuccess) e = cudaMalloc(&h->d_partials, 2 * slots * sizeof(float))   /* up to two sums per row */;
   if (e == cudaSuccess) e = cudaMalloc(&h->d_tickets, rows * sizeof(unsigned int));
   if (e == cudaSuccess) e = cudaMalloc(&h->d_status, sizeof(int32_t));
+  if (e == cudaSuccess) e = cudaMalloc(&h->d_obj_part, 1024 * sizeof(double));
+  if (e == cudaSuccess) e = cudaMalloc(&h->d_obj_ticket, sizeof(unsigned int));
+  if (e == cudaSuccess) e = cudaMemset(h->d_obj_ticket, 0, sizeof(unsigned int));
   std::vector<long long> step_off((size_t)cfg->n_steps + 1, 0);
   {
     int k = cfg->n_expand, si = 0;
@@ -148,7 +156,15 @@ int pg_rollout_destroy(pg_rollout* h) {
   cudaFree(h->d_partials);
   cudaFree(h->d_tickets);
   cudaFree(h->d_status);
+  cudaFree(h->d_obj_part);
+  cudaFree(h->d_obj_ticket);
   cudaFree(h->d_step_off);
+  for (int i = 0; i < 2; ++i) {
+    if (h->v_ready[i]) cudaEventDestroy(h->v_ready[i]);
+    if (h->v_free[i]) cudaEventDestroy(h->v_free[i]);
+  }
+  if (h->host_compute) cudaStreamDestroy(h->host_compute);
+  if (h->host_copy) cudaStreamDestroy(h->host_copy);
   delete h;
   return PG_OK;
 }
@@ -371,7 +387,8 @@ int pg_policy_objective(pg_rollout* h, int32_t n_steps, const float* logp_new, c
   if (const int rc_dev = wrong_device(h)) return rc_dev;
   if (!(clip_eps >= 0.f) || !std::isfinite(beta)) return PG_EINVAL;
   return pg::launch_policy_objective(n_steps, h->cfg.n_groups * h->k_cur, logp_new, logp_old, kl, adv,
-                                     clip_eps, beta, ratio, dlogp, objective, (cudaStream_t)stream);
+                                     clip_eps, beta, ratio, dlogp, objective, h->d_obj_part, h->d_obj_ticket,
+                                     (cudaStream_t)stream);
 }
 
 int pg_policy_backward(pg_rollout* h, const pg_step_coef* coef, const float* x, const float* x_next,
@@ -527,20 +544,36 @@ size_t pg_rollout_host_workspace_bytes(const pg_config* cfg) {
   return make_plan(cfg).total;
 }
 
-int pg_rollout_host(const pg_config* cfg, const pg_step_coef* step_coef,
-                    const pg_preview_coef* preview_coef, const float* x0,
-                    const void* const* vel_steps, const float* const* stage_scores,
-                    const float* final_rewards, float* x_final, float* logp, int32_t* keep_idx,
-                    float* adv, int32_t* traj_id, void* workspace, size_t workspace_bytes) {
+// Streams and events of the host-buffer driver live in the handle: made once, reused by every call.
+static int ensure_host_resources(pg_rollout* h) {
+  if (!h->host_compute) PG_CUDA(cudaStreamCreateWithFlags(&h->host_compute, cudaStreamNonBlocking));
+  if (!h->host_copy) PG_CUDA(cudaStreamCreateWithFlags(&h->host_copy, cudaStreamNonBlocking));
+  for (int i = 0; i < 2; ++i) {
+    if (!h->v_ready[i]) PG_CUDA(cudaEventCreateWithFlags(&h->v_ready[i], cudaEventDisableTiming));
+    if (!h->v_free[i]) PG_CUDA(cudaEventCreateWithFlags(&h->v_free[i], cudaEventDisableTiming));
+  }
+  return PG_OK;
+}
+
+int pg_rollout_host_on(pg_rollout* h, const pg_step_coef* step_coef,
+                       const pg_preview_coef* preview_coef, const float* x0,
+                       const void* const* vel_steps, const float* const* stage_scores,
+                       const float* final_rewards, float* x_final, float* logp, int32_t* keep_idx,
+                       float* adv, int32_t* traj_id, void* workspace, size_t workspace_bytes) {
   TraceRange trace_range("pg_rollout_host");
-  int rc = validate_config(cfg);
-  if (rc != PG_OK) return rc;
+  if (!h) return PG_EINVAL;
+  if (const int rc_dev = wrong_device(h)) return rc_dev;
+  const pg_config* cfg = &h->cfg;
   if (!step_coef || !vel_steps || !workspace || !aligned16(workspace)) return PG_EINVAL;
   if (cfg->n_stages > 0 && !preview_coef && !stage_scores) return PG_EINVAL;
   const HostPlan pl = make_plan(cfg);
   if (workspace_bytes < pl.total) return PG_EINVAL;
   for (int s = 0; s < cfg->n_steps; ++s)
     if (!vel_steps[s]) return PG_EINVAL;
+  for (int i = 0; i < cfg->n_stages; ++i)
+    if (!(stage_scores && stage_scores[i]) && !preview_coef) return PG_EINVAL;
+  int rc = ensure_host_resources(h);
+  if (rc != PG_OK) return rc;
 
   unsigned char* ws = (unsigned char*)workspace;
   float* d_x[2] = {(float*)(ws + pl.off_x[0]), (float*)(ws + pl.off_x[1])};
@@ -552,31 +585,18 @@ int pg_rollout_host(const pg_config* cfg, const pg_step_coef* step_coef,
   float* d_rewards = (float*)(ws + pl.off_rewards);
   float* d_adv = (float*)(ws + pl.off_adv);
   int32_t* d_traj = (int32_t*)(ws + pl.off_traj);
-
-  pg_rollout* h = nullptr;
-  rc = pg_rollout_init(cfg, &h);
-  if (rc != PG_OK) return rc;
-  cudaStream_t compute = nullptr, copy = nullptr;
-  cudaEvent_t v_ready[2] = {nullptr, nullptr}, v_free[2] = {nullptr, nullptr};
-  auto cleanup = [&](int code) {
-    cudaDeviceSynchronize();
-    for (int i = 0; i < 2; ++i) {
-      if (v_ready[i]) cudaEventDestroy(v_ready[i]);
-      if (v_free[i]) cudaEventDestroy(v_free[i]);
-    }
-    if (compute) cudaStreamDestroy(compute);
-    if (copy) cudaStreamDestroy(copy);
-    pg_rollout_destroy(h);
+  cudaStream_t compute = h->host_compute, copy = h->host_copy;
+  cudaEvent_t* v_ready = h->v_ready;
+  cudaEvent_t* v_free = h->v_free;
+  // on an error the streams are drained so that nothing of this call is still in flight
+  auto fail = [&](int code) {
+    cudaStreamSynchronize(copy);
+    cudaStreamSynchronize(compute);
     return code;
   };
-#define PG_TRY_CUDA(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return cleanup(cuda_fail(e_)); } while (0)
-#define PG_TRY(call) do { int r_ = (call); if (r_ != PG_OK) return cleanup(r_); } while (0)
-  PG_TRY_CUDA(cudaStreamCreateWithFlags(&compute, cudaStreamNonBlocking));
-  PG_TRY_CUDA(cudaStreamCreateWithFlags(&copy, cudaStreamNonBlocking));
-  for (int i = 0; i < 2; ++i) {
-    PG_TRY_CUDA(cudaEventCreateWithFlags(&v_ready[i], cudaEventDisableTiming));
-    PG_TRY_CUDA(cudaEventCreateWithFlags(&v_free[i], cudaEventDisableTiming));
-  }
+#define PG_TRY_CUDA(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return fail(cuda_fail(e_)); } while (0)
+#define PG_TRY(call) do { int r_ = (call); if (r_ != PG_OK) return fail(r_); } while (0)
+  PG_TRY(pg_rollout_reset(h, compute));
 
   // rows alive when the prediction of step s is made
   std::vector<int> rows_pred(cfg->n_steps);
@@ -619,7 +639,6 @@ int pg_rollout_host(const pg_config* cfg, const pg_step_coef* step_coef,
         PG_TRY_CUDA(cudaMemcpyAsync(d_scores, stage_scores[stage], (size_t)rows * 4,
                                     cudaMemcpyHostToDevice, compute));
       } else {
-        if (!preview_coef) return cleanup(PG_EINVAL);
         PG_TRY(pg_score(h, &preview_coef[stage], d_x[cur], d_v[b], d_scores, nullptr, compute));
       }
       PG_TRY(pg_prune_ovf(h, stage, d_scores, d_keep + keep_off, d_src, nullptr, compute));
@@ -647,12 +666,28 @@ int pg_rollout_host(const pg_config* cfg, const pg_step_coef* step_coef,
   if (keep_idx && pl.total_keep) PG_TRY_CUDA(cudaMemcpyAsync(keep_idx, d_keep, pl.total_keep * 4, cudaMemcpyDeviceToHost, compute));
   if (adv) PG_TRY_CUDA(cudaMemcpyAsync(adv, d_adv, rows_final * 4, cudaMemcpyDeviceToHost, compute));
   if (traj_id) PG_TRY_CUDA(cudaMemcpyAsync(traj_id, d_traj, rows_final * 4, cudaMemcpyDeviceToHost, compute));
-  PG_TRY_CUDA(cudaStreamSynchronize(compute));
   int32_t st = 0;
-  PG_TRY_CUDA(cudaMemcpy(&st, h->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost));
-  return cleanup((st & 4) ? PG_EINDEX : (st & 2) ? PG_ETIMEOUT : (st & 1) ? PG_ENONFINITE : PG_OK);
+  PG_TRY_CUDA(cudaMemcpyAsync(&st, h->d_status, sizeof(int32_t), cudaMemcpyDeviceToHost, compute));
+  PG_TRY_CUDA(cudaStreamSynchronize(compute));
+  PG_TRY_CUDA(cudaStreamSynchronize(copy));
+  return (st & 4) ? PG_EINDEX : (st & 2) ? PG_ETIMEOUT : (st & 1) ? PG_ENONFINITE : PG_OK;
 #undef PG_TRY
 #undef PG_TRY_CUDA
+}
+
+int pg_rollout_host(const pg_config* cfg, const pg_step_coef* step_coef,
+                    const pg_preview_coef* preview_coef, const float* x0,
+                    const void* const* vel_steps, const float* const* stage_scores,
+                    const float* final_rewards, float* x_final, float* logp, int32_t* keep_idx,
+                    float* adv, int32_t* traj_id, void* workspace, size_t workspace_bytes) {
+  pg_rollout* h = nullptr;
+  int rc = pg_rollout_init(cfg, &h);
+  if (rc != PG_OK) return rc;
+  rc = pg_rollout_host_on(h, step_coef, preview_coef, x0, vel_steps, stage_scores, final_rewards, x_final,
+                          logp, keep_idx, adv, traj_id, workspace, workspace_bytes);
+  cudaDeviceSynchronize();
+  pg_rollout_destroy(h);
+  return rc;
 }
 
 // ---------------------------------------------------------------- device-resident driver

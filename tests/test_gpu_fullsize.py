@@ -1,6 +1,7 @@
 """Full-size parity: the large workload exactly as bench.py launches it (64 groups x 64
-trajectories, d = 262144, bf16 predictions generated on the device), checked against the oracle
-on sampled prompt groups followed end to end, plus whole-batch properties."""
+trajectories, d = 262144, bf16 predictions generated on the device), every one of its 64 prompt
+groups followed end to end by the oracle (streamed through the host eight groups at a time), plus
+whole-batch properties."""
 import numpy as np
 import pytest
 import torch
@@ -11,10 +12,10 @@ from tests import util as U
 
 pytestmark = pytest.mark.gpu
 
-SAMPLED_GROUPS = (0, 5, 17, 31, 37, 50, 62, 63)
+GROUP_BATCH = 8          # groups whose predictions are held on the host at a time (2.8 GB)
 
 
-def test_large_workload_sampled_groups_match_oracle():
+def test_large_workload_every_group_matches_oracle():
     from paper_2512_15347_b200 import binding as B
     from paper_2512_15347_b200.rollout import Rollout
     w = wl.WORKLOADS["large"]
@@ -25,16 +26,9 @@ def test_large_workload_sampled_groups_match_oracle():
     ro = Rollout(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, torch.bfloat16,
                  adv_eps=w.adv_eps)
     x0 = wl.initial_latents(w, device=dev)
-    host_x0 = {g: x0[g * w.n_expand:(g + 1) * w.n_expand].cpu().numpy() for g in SAMPLED_GROUPS}
-    host_vel = {g: [] for g in SAMPLED_GROUPS}
 
     def velocity(s, x_active):
-        rows = w.n_groups * w.rows_before(s)
-        v = wl.normal_velocity(w, s, rows, device=dev)
-        per = w.rows_before(s)
-        for g in SAMPLED_GROUPS:
-            host_vel[g].append(wl.as_numpy_velocity(v[g * per:(g + 1) * per]))
-        return v
+        return wl.normal_velocity(w, s, w.n_groups * w.rows_before(s), device=dev)
 
     out = ro.run(x0, w.step_coef, w.preview_coef, velocity, record_scores=True)
     torch.cuda.synchronize()
@@ -63,29 +57,59 @@ def test_large_workload_sampled_groups_match_oracle():
         lp = out.logp[s].cpu().numpy().astype(np.float64)
         assert abs(lp.mean() - want) < 6 * np.sqrt(w.elems / 2) / np.sqrt(lp.size)
 
-    # sampled groups: the oracle follows each group through the whole schedule
+    # every group: the oracle follows it through the whole schedule.  The predictions are seeded per
+    # step, so they are generated again on the device and the groups' slices copied to the host.
     k_final = w.final_keep
-    for g in SAMPLED_GROUPS:
-        ref = oracle.rollout(host_x0[g], 1, w.n_expand, w.n_steps, w.stages, w.seed, w.step_coef,
-                             w.preview_coef, lambda s, x, traj, g=g: host_vel[g][s],
-                             adv_eps=w.adv_eps, group_offset=g)
-        k_prev = w.n_expand
-        for i, (s, k) in enumerate(w.stages):
-            got_sc = out.stage_scores[i].cpu().numpy().reshape(w.n_groups, k_prev)[g]
-            assert np.abs(got_sc.astype(np.float64) - ref.stage_scores[i][0]).max() <= U.SCORE_GAP
-            np.testing.assert_array_equal(out.stage_keep[i].cpu().numpy().reshape(w.n_groups, k)[g],
-                                          ref.stage_keep[i][0])
-            k_prev = k
+    got_scores = [t.cpu().numpy() for t in out.stage_scores]
+    got_keep = [t.cpu().numpy() for t in out.stage_keep]
+    got_logp = [t.cpu().numpy() for t in out.logp]
+    got_adv = out.adv.cpu().numpy().reshape(w.n_groups, k_final)
+    got_ids = out.traj_id.cpu().numpy()
+    diverged = []
+    worst_lp = worst_x = 0.0
+    for b0 in range(0, w.n_groups, GROUP_BATCH):
+        groups = range(b0, min(b0 + GROUP_BATCH, w.n_groups))
+        host_vel = {g: [] for g in groups}
         for s in range(w.n_steps):
-            per = w.active_at(s)
-            got = out.logp[s].cpu().numpy()[g * per:(g + 1) * per]
-            assert U.logp_err(got, ref.logp[s], w.elems) <= U.LOGP_TOL
-        got_x = out.x_final[g * k_final:(g + 1) * k_final].cpu().numpy()
-        assert U.latent_err(got_x, ref.x_final) <= U.LATENT_TOL
-        np.testing.assert_array_equal(out.traj_id.cpu().numpy()[g * k_final:(g + 1) * k_final],
-                                      ref.traj_id)
-        np.testing.assert_allclose(out.adv.cpu().numpy().reshape(w.n_groups, k_final)[g], ref.adv[0],
-                                   rtol=2e-4, atol=2e-5)
+            per = w.rows_before(s)
+            v = wl.normal_velocity(w, s, w.n_groups * per, device=dev)
+            for g in groups:
+                host_vel[g].append(wl.as_numpy_velocity(v[g * per:(g + 1) * per]))
+            del v
+        for g in groups:
+            host_x0 = x0[g * w.n_expand:(g + 1) * w.n_expand].cpu().numpy()
+            ref = oracle.rollout(host_x0, 1, w.n_expand, w.n_steps, w.stages, w.seed, w.step_coef,
+                                 w.preview_coef, lambda s, x, traj, g=g: host_vel[g][s],
+                                 adv_eps=w.adv_eps, group_offset=g)
+            k_prev = w.n_expand
+            same_until = w.n_steps          # first step at which the survivors differ from the oracle's
+            for i, (s, k) in enumerate(w.stages):
+                if s >= same_until:
+                    break
+                sc = got_scores[i].reshape(w.n_groups, k_prev)[g]
+                assert np.abs(sc.astype(np.float64) - ref.stage_scores[i][0]).max() <= U.SCORE_GAP
+                if not np.array_equal(got_keep[i].reshape(w.n_groups, k)[g], ref.stage_keep[i][0]):
+                    # scores agree within the tolerance and the selection is the oracle's on the
+                    # device's own scores (checked above for the whole batch): a near-tie
+                    same_until = s
+                    diverged.append(g)
+                k_prev = k
+            for s in range(min(same_until, w.n_steps)):
+                per = w.active_at(s)
+                e = U.logp_err(got_logp[s][g * per:(g + 1) * per], ref.logp[s], w.elems)
+                worst_lp = max(worst_lp, e)
+                assert e <= U.LOGP_TOL, (g, s, e)
+            if same_until < w.n_steps:
+                continue
+            e = U.latent_err(out.x_final[g * k_final:(g + 1) * k_final].cpu().numpy(), ref.x_final)
+            worst_x = max(worst_x, e)
+            assert e <= U.LATENT_TOL, (g, e)
+            np.testing.assert_array_equal(got_ids[g * k_final:(g + 1) * k_final], ref.traj_id)
+            np.testing.assert_allclose(got_adv[g], ref.adv[0], rtol=2e-4, atol=2e-5)
+        del host_vel
+    assert len(diverged) <= w.n_groups // 10, diverged      # near-ties are rare
+    print(f"large workload: 64 groups followed, worst log-prob err {worst_lp:.2e}, latent err {worst_x:.2e}, "
+          f"near-tie groups {diverged}")
     ro.close()
 
 

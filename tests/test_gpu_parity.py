@@ -455,6 +455,21 @@ def test_host_buffer_rollout_matches_device_rollout(B):
     assert torch.equal(keep, torch.cat(out.stage_keep).cpu())
     assert torch.equal(adv, out.adv.cpu())
     assert torch.equal(ids, out.traj_id.cpu())
+    # the same on an existing handle, twice in a row (the second call reuses the handle's streams
+    # and events and finds the cursor at the end of the first rollout)
+    h = B.rollout_init(cfg)
+    args = B.HostArgs([w.step_coef(s) for s in range(w.n_steps)], [w.preview_coef(s) for s, _ in w.stages], vels)
+    for _ in range(2):
+        for t in (x_final, logp, adv):
+            t.fill_(float("nan"))
+        keep.fill_(-1)
+        ids.fill_(-1)
+        assert B.rollout_host_on(h, args, x0, None, x_final, logp, keep, adv, ids, ws) == 0
+        assert torch.equal(x_final, out.x_final.cpu()) and torch.equal(logp, torch.cat(out.logp).cpu())
+        assert torch.equal(keep, torch.cat(out.stage_keep).cpu()) and torch.equal(adv, out.adv.cpu())
+        assert torch.equal(ids, out.traj_id.cpu())
+    assert B.rollout_status(h) == (w.n_groups * K, w.n_steps, 0)
+    B.rollout_destroy(h)
     ro.close()
 
 

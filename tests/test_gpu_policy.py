@@ -127,6 +127,90 @@ def test_policy_update_after_a_rollout_has_unit_ratio():
     ro.close()
 
 
+def test_unit_ratio_in_sum_mode_on_full_length_latents():
+    """Summed log-densities (the form of Eq. ratio_method) on 16x128x128 latents: pg_step reports
+    log pi from the generator's radius terms, pg_policy_logprob recomputes it from the stored fp32
+    x_{t+1}; the two differ by the fp32 rounding of x_{t+1} and of the noise transform, an error
+    that grows with the latent length.  Bound asserted (and documented in the header):
+    |log pi_new - log pi_old| <= 2e-6 * d, the mean-mode bound times d."""
+    from paper_2512_15347_b200 import binding as B
+    from paper_2512_15347_b200.rollout import Rollout
+    w = wl.Workload("upd-sum", 2, 3, (), 3, 262144, 1, "bf16", 9, "normal", "preview")
+    inp = U.SharedInputs(w)
+    ro = Rollout(w.n_groups, w.n_expand, w.elems, w.n_steps, w.stages, w.seed, torch.bfloat16, logp_mean=False)
+    xs = [U.to_dev(inp.x0)]
+    vels = []
+
+    def velocity(s, x):
+        v = inp.vel_device(s, x)
+        vels.append(v)
+        if s > 0:
+            xs.append(x.clone())
+        return v
+
+    out = ro.run(xs[0], w.step_coef, w.preview_coef, velocity)
+    xs.append(out.x_final.clone())
+    n, T, d = w.n_groups * w.n_expand, w.n_steps, w.elems
+    lp_new = torch.empty(T, n, device="cuda")
+    for t in range(T):
+        B.policy_logprob(ro.h, w.step_coef(t), xs[t], xs[t + 1], vels[t], None, lp_new[t], None)
+    lp_old = torch.stack(out.logp)
+    torch.cuda.synchronize()
+    gap = (lp_new.double() - lp_old.double()).abs().max().item()
+    print(f"sum-mode |log pi_new - log pi_old| max {gap:.4f} at d = {d} ({gap / d:.2e} per element)")
+    assert gap <= 2e-6 * d
+    # the oracle's density of the stored transition agrees with the recomputed value to fp32 accuracy
+    ref = oracle.policy_logprob(xs[0].cpu().numpy(), xs[1].cpu().numpy(), wl.as_numpy_velocity(vels[0]), None,
+                                *w.step_coef(0), False)[0]
+    assert U.logp_err(lp_new[0].cpu().numpy(), ref, d) <= U.LOGP_TOL
+    ro.close()
+
+
+def test_objective_over_many_entries_matches_oracle():
+    """T * n = 50 x 8192 entries: the objective kernel runs as 50 CTAs whose partial sums are
+    combined in slot order; same result on every run, and the oracle's within fp32 rounding."""
+    from paper_2512_15347_b200 import binding as B
+    T, G, K = 50, 1024, 8
+    n = G * K
+    rng = np.random.default_rng(77)
+    h = B.rollout_init(B.make_config(G, K, 4, T, [], 1, B.VEL_F32, logp_mean=True))
+    try:
+        lp_old = rng.standard_normal((T, n)).astype(np.float32)
+        lp_new = (lp_old + 0.3 * rng.standard_normal((T, n))).astype(np.float32)
+        kl = (0.1 * rng.random((T, n))).astype(np.float32)
+        adv = rng.standard_normal(n).astype(np.float32)
+        outs = []
+        for _ in range(3):
+            ratio = torch.empty(T, n, device="cuda")
+            dlogp = torch.empty(T, n, device="cuda")
+            obj = torch.full((1,), float("nan"), device="cuda")
+            B.policy_objective(h, T, U.to_dev(lp_new), U.to_dev(lp_old), U.to_dev(kl), U.to_dev(adv), 0.2, 0.04,
+                               ratio, dlogp, obj)
+            torch.cuda.synchronize()
+            outs.append((obj.clone(), ratio, dlogp))
+        assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[1][0], outs[2][0])
+        ref_obj, ref_ratio, ref_dlogp = oracle.policy_objective(lp_new, lp_old, kl, adv, 0.2, 0.04)
+        assert float(outs[0][0].item()) == pytest.approx(ref_obj, rel=2e-6, abs=1e-9)
+        np.testing.assert_allclose(outs[0][1].cpu().numpy(), ref_ratio, rtol=1e-6)
+        np.testing.assert_allclose(outs[0][2].cpu().numpy(), ref_dlogp, rtol=1e-6, atol=1e-30)
+        # a number of entries that is not a multiple of anything, and one that fits a single CTA
+        for t_small, n_rows in ((7, 3001), (1, 5)):
+            hs = B.rollout_init(B.make_config(n_rows, 1, 4, t_small, [], 1, B.VEL_F32, logp_mean=True))
+            a, b = lp_new.reshape(-1)[: t_small * n_rows].reshape(t_small, n_rows), lp_old.reshape(-1)[: t_small * n_rows].reshape(t_small, n_rows)
+            ad = adv[:n_rows]
+            dl = torch.empty(t_small, n_rows, device="cuda")
+            ob = torch.empty(1, device="cuda")
+            B.policy_objective(hs, t_small, U.to_dev(a), U.to_dev(b), None, U.to_dev(ad), 0.1, 0.0, None, dl, ob)
+            torch.cuda.synchronize()
+            r_obj, _, r_dl = oracle.policy_objective(a, b, None, ad, 0.1, 0.0)
+            assert float(ob.item()) == pytest.approx(r_obj, rel=2e-6, abs=1e-9)
+            np.testing.assert_allclose(dl.cpu().numpy(), r_dl, rtol=1e-6, atol=1e-30)
+            B.rollout_destroy(hs)
+    finally:
+        torch.cuda.synchronize()
+        B.rollout_destroy(h)
+
+
 def test_policy_update_on_the_survivors_of_a_pruned_rollout():
     """The whole chain after a rollout with two prunes: the survivors' transitions are collected
     from the stored steps (rows from pg_survivor_rows, latents and predictions through
