@@ -359,7 +359,8 @@ def _other_workload(name, dev, reps, peak):
 LAUNCH_ROWS = (192, 384, 768, 1024, 2048, 4096)
 
 
-def launch_size_table(B, x_a, x_b, vel, elems, peak, rows_list=LAUNCH_ROWS, reps=24):
+def launch_size_table(B, x_a, x_b, vel, elems, peak, rows_list=LAUNCH_ROWS, reps=24,
+                      step_coef=(1.0, 0.04, 0.13)):
     """Step and score launches of the streaming shape (d = `elems`, bf16 predictions) by row count:
     device time per launch and algorithmic GB/s, measured two ways - `stream`: `reps` launches
     enqueued back to back between one pair of CUDA events (how a rollout issues them; successive
@@ -380,7 +381,7 @@ def launch_size_table(B, x_a, x_b, vel, elems, peak, rows_list=LAUNCH_ROWS, reps
 
         def step(i):
             o = (i * rows) % span
-            B.step(h, nxt[0], (1.0, 0.04, 0.13), x_a[o:o + rows], vel[o:o + rows], None, x_b[o:o + rows], lp)
+            B.step(h, nxt[0], step_coef, x_a[o:o + rows], vel[o:o + rows], None, x_b[o:o + rows], lp)
             nxt[0] += 1
 
         def score(i):
@@ -650,14 +651,47 @@ def run_ours(args):
         xs, vs = ro.x[0][:rows_out], vels[0][:rows_out]
         out16 = torch.empty(rows_out, w.elems, device=dev, dtype=torch.bfloat16)
         t_p16 = timed(lambda: B.preview(hp, (1.0, 0.5), xs, vs, out16))
+        # scores and the bf16 preview in one pass (what a decoder + reward model between preview and
+        # selection need), against scoring alone and against the two separate passes
+        sc_out = torch.empty(rows_out, device=dev)
+        t_sp16 = timed(lambda: B.score_preview(hp, (1.0, 0.5), xs, vs, sc_out, out16))
+        t_s = timed(lambda: B.score(hp, (1.0, 0.5), xs, vs, sc_out))
         del out16
         B.rollout_destroy(hp)
         other = {"compact_gbs": rows_out * w.elems * 8 / (t_c * 1e-3) / 1e9,
                  "compact_rows": [rows_in, rows_out],
                  "preview_bf16_gbs": rows_out * w.elems * 8 / (t_p16 * 1e-3) / 1e9,
-                 "bytes_per_element": {"compact": 8, "preview_bf16": 8},
+                 "score_preview_bf16_gbs": rows_out * w.elems * 8 / (t_sp16 * 1e-3) / 1e9,
+                 "score_preview_bf16_frac_of_peak": rows_out * w.elems * 8 / (t_sp16 * 1e-3) / 1e9 / peak,
+                 "score_preview_bf16_us": t_sp16 * 1e3, "score_then_preview_us": (t_s + t_p16) * 1e3,
+                 "bytes_per_element": {"compact": 8, "preview_bf16": 8, "score_preview_bf16": 8,
+                                       "score_then_preview": 14},
                  "note": "pg_compact gathers the first stage's survivors (fp32 rows); pg_preview writes "
-                         "the bf16 look-ahead latent for an external decoder"}
+                         "the bf16 look-ahead latent for an external decoder; pg_score_preview does the "
+                         "scoring pass and that emission in one pass over (x, v)"}
+
+    # the same rollout under the coefficients of the diffusion branch (DDIM over the linear-beta
+    # schedule: c_x != 1, so every step takes the step kernel's general-coefficient variant)
+    general = None
+    if rank == 0 and w.velocity == "normal":
+        from dataclasses import replace as _replace
+        wg = _replace(w, coef="ddim", eta=1.0)
+        gen_run = lambda trace=None: ro.run(x0, wg.step_coef, wg.preview_coef, velocity, external_scores=ext,
+                                            final_rewards=fin, trace=trace)
+        gen_run()
+        torch.cuda.synchronize()
+        gtr = []
+        for _ in range(min(args.steps, 5)):
+            tr = []
+            gen_run(trace=tr)
+            gtr.append(tr)
+        torch.cuda.synchronize()
+        g_ms = sum(a.elapsed_time(b) for tr in gtr for kind, _, a, b in tr if kind == "step")
+        g_rows = sum(rows for tr in gtr for kind, rows, _, _ in tr if kind == "step")
+        g_gbs = g_rows * (w.elems * (8 + vel_bytes) + 4) / (g_ms * 1e-3) / 1e9
+        general = {"kernel": "step_kernel<general coefficients> (c_x != 1: DDIM schedule, eta = 1; last step deterministic)",
+                   "step_gbs": g_gbs, "step_frac_of_peak": g_gbs / peak,
+                   "unit_cx_step_gbs": step_gbs, "rollouts": len(gtr)}
 
     # step / score launches by row count on the streaming shape
     by_rows = None
@@ -702,7 +736,8 @@ def run_ours(args):
                                 v["launches"] // args.steps} for k, v in kinds.items()},
                 "score_gbs": score_gbs, "prune_stage_gbs": prune_stage_gbs,
                 "hbm_gbs_whole_rollout": (step_bytes + (score_bytes if score_gbs else 0)) / (total_ms * 1e-3) / 1e9,
-                "ovf_microbench": ovf, "drivers": drivers, "policy_update": policy, "other_kernels": other, "launch_size_table": by_rows, "other_workloads": others, "e2e": e2e, "cpu_baseline": cpu_base}
+                "ovf_microbench": ovf, "drivers": drivers, "policy_update": policy, "other_kernels": other, "general_coefficients": general,
+                "launch_size_table": by_rows, "other_workloads": others, "e2e": e2e, "cpu_baseline": cpu_base}
         if gathered is not None:
             line["gathered"] = gathered
         print(json.dumps(line))

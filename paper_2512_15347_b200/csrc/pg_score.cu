@@ -55,8 +55,11 @@ template <> struct EmitType<kEmitBf16> { using type = __nv_bfloat16; };
 
 constexpr int kScoreUnroll = 4;   // quads per thread and iteration (loads of the next batch in flight)
 
+// The bf16-prediction variants that also write the preview are held to 64 registers (four CTAs per SM, like the
+// scoring-only variants): at the 69 - 70 registers the compiler would otherwise take, three CTAs
+// fit and the bf16-emitting pass measured 6.47 instead of 6.82 TB/s on 2048 rows of 262144.
 template <typename VelT, bool kUseVel, int kEmit>
-__global__ void __launch_bounds__(kRowThreads)
+__global__ void __launch_bounds__(kRowThreads, (kEmit != kEmitNone && sizeof(VelT) == 2) ? 4 : 0)
 score_kernel(const __grid_constant__ ScoreParams p) {
   using Raw = typename VelRaw<VelT>::type;
   using OutT = typename EmitType<kEmit>::type;
