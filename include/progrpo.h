@@ -254,6 +254,11 @@ int pg_advantages(pg_rollout *h, const float *rewards, float *adv, float *mean, 
  * [n_active, d] in cfg.vel_dtype: new and reference predictions.  vel_ref and kl_out are
  * both NULL or both given.  Read-only pass; uses the handle's reduction scratch (same stream
  * rule as the other calls).  Does not move any cursor.
+ * At the rollout's own prediction this is pg_step's logp_out up to fp32 rounding: pg_step reports
+ * the density of the sampled action from the generator's radius terms, this call recomputes it
+ * from the stored fp32 x_next, and the two differ by at most 2e-6 * d in sum mode (2e-6 with
+ * logp_mean) - 0.5 for a 262144-element latent.  Ratios pi_theta / pi_old that must be exactly 1 at
+ * theta_old should take both log-probs from this call, or use logp_mean.
  */
 int pg_policy_logprob(pg_rollout *h, const pg_step_coef *coef, const float *x, const float *x_next,
                       const void *vel, const void *vel_ref, float *logp_out, float *kl_out, void *stream);

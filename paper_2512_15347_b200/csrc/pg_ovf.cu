@@ -200,6 +200,8 @@ ovf_warp_kernel(const __grid_constant__ OvfParams p, int n_groups) {
       uint32_t other[E];
 #pragma unroll
       for (int r = 0; r < E; ++r) other[r] = __shfl_xor_sync(kFull, key[r ^ (E - 1)], lane_mask);
+      // (a compare combined with the lane's side plus one select instead of min, max and select
+      // measured slower: 15.1 instead of 13.8 us on 4096 groups of 256)
 #pragma unroll
       for (int r = 0; r < E; ++r) key[r] = lower ? min(key[r], other[r]) : max(key[r], other[r]);
     }
