@@ -88,16 +88,14 @@ __device__ __forceinline__ float box_muller(uint32_t r0, uint32_t r1, float& rad
   neg2ln = (w < 0.015625f) ? ser : neg2ln;
   asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(radius) : "f"(neg2ln));
   const float turn = fmaf((float)(r1 >> 8), 5.9604644775390625e-8f, -0.5f);  // u2 - 1/2, exact
-  // The cosine is taken as the sine of the angle a quarter turn further, wrapped back into
-  // [-1/2, 1/2) turns (all exact on the 24-bit grid).  The hardware sine's error is an odd
-  // function of the angle, so over the symmetric angle grid it averages to zero; the hardware
-  // cosine's error is even and does not (measured mean +5.8e-8, i.e. -7.2e-8 on every cosine
-  // normal) - small against the 2e-7 rms error of a draw, but a bias is what the mean of a long
-  // latent (the latent score) accumulates over many steps.
-  float turn_c = turn + 0.25f;
-  turn_c = turn_c >= 0.5f ? turn_c - 1.0f : turn_c;
+  // The cosine is taken as a sine: cos t = sin(pi/2 - |t|), i.e. the sine at 1/4 - |turn| turns
+  // (an exact difference on the 24-bit grid, and an argument in [-pi/2, pi/2]).  The hardware
+  // sine's error is an odd function of the angle, so over the symmetric angle grid it averages to
+  // zero; the hardware cosine's error is even and does not (measured mean +5.8e-8, i.e. -7.2e-8
+  // on every cosine normal) - small against the 2e-7 rms error of a draw, but a bias is what the
+  // mean of a long latent (the latent score) accumulates over many steps.
   const float angle = 6.283185307179586f * turn;
-  const float angle_c = 6.283185307179586f * turn_c;
+  const float angle_c = 6.283185307179586f * (0.25f - fabsf(turn));
   asm("sin.approx.ftz.f32 %0, %1;" : "=f"(s) : "f"(angle));
   asm("sin.approx.ftz.f32 %0, %1;" : "=f"(c) : "f"(angle_c));
   return neg2ln;
