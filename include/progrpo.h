@@ -339,7 +339,8 @@ int pg_rollout_host(const pg_config *cfg, const pg_step_coef *step_coef,
  * handle is rewound first; its two streams and four events are created on the first call and
  * released by pg_rollout_destroy, so later calls allocate nothing.  Arguments, layout of the
  * outputs and the workspace are those of pg_rollout_host (schedule = the handle's); synchronises
- * before returning.
+ * before returning.  The work runs on the handle's own streams: the handle must be idle when
+ * the call is made (nothing enqueued on it by the caller still in flight).
  */
 int pg_rollout_host_on(pg_rollout *h, const pg_step_coef *step_coef,
                        const pg_preview_coef *preview_coef, const float *x0,

@@ -32,6 +32,7 @@ def test_reference_arm_prints_one_line_with_the_contract_keys():
     assert "workload" in d["config"] and d["config"]["workload"].startswith("sd15")
     cb = d["cpu_baseline"]
     assert cb["kind"] == "oracle" and cb["cores"] >= 1 and cb["sample"] and cb["value"] == d["value"]
+    assert isinstance(cb["cpu_model"], str) and cb["cpu_model"]
     e = d["e2e"]
     assert e["value"] == d["value"] and e["unit"] == d["unit"]
     assert e["h2d_bytes_per_step"] == 0 and e["d2h_bytes_per_step"] == 0
@@ -55,8 +56,11 @@ def test_gpu_arm_prints_roofline_baseline_and_end_to_end():
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and r["peak"] > 0 and r["achieved"] > 0
     assert abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9 and "traffic" in r
+    # the prune stage (scoring pass + selection) is in the record next to the step kernel
+    stage = [a for a in r["also"] if a["kernel"].startswith("score + ovf")]
+    assert len(stage) == 1 and stage[0]["achieved"] > 0 and abs(stage[0]["frac"] - stage[0]["achieved"] / r["peak"]) < 1e-9
     cb = d["cpu_baseline"]
-    assert cb["kind"] == "oracle" and cb["value"] > 0 and cb["cores"] >= 1 and cb["sample"]
+    assert cb["kind"] == "oracle" and cb["value"] > 0 and cb["cores"] >= 1 and cb["sample"] and cb["cpu_model"]
     e = d["e2e"]
     assert e["value"] > 0 and e["h2d_bytes_per_step"] > 0 and e["d2h_bytes_per_step"] > 0
     assert e["value"] != d["value"]

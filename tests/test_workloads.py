@@ -41,3 +41,39 @@ def test_score_distributions_have_the_stated_structure():
     w = wl.WORKLOADS["large"]
     assert [w.active_at(s) for s in (0, 1, 2, 4, 5, 7, 8, 27)] == [64, 64, 32, 32, 16, 16, 16, 16]
     assert [w.rows_before(s) for s in (0, 2, 3, 5, 6, 8, 9)] == [64, 64, 32, 32, 16, 16, 16]
+
+
+def test_traffic_ratio_follows_the_committed_profile_and_the_kernel_sources(tmp_path):
+    """bench.py takes roofline.traffic from the ncu summary under profiles/ and drops it as soon as
+    the kernel sources no longer hash to the value recorded there."""
+    import bench
+    prof = tmp_path / "step.txt"
+    prof.write_text("source_sha256: " + bench._sources_sha256() + "\nalgorithmic_bytes: 1000\n"
+                    "  dram__bytes_read.sum    0.600 Kbyte\n  dram__bytes_write.sum   300 byte\n")
+    ratio, note = bench.step_traffic_ratio(str(prof))
+    assert abs(ratio - 0.9) < 1e-12
+    prof.write_text(prof.read_text().replace(bench._sources_sha256(), "0" * 64))
+    assert bench.step_traffic_ratio(str(prof))[0] is None
+    assert bench.step_traffic_ratio(str(tmp_path / "missing.txt"))[0] is None
+    assert isinstance(bench.cpu_model(), str) and bench.cpu_model()
+
+
+def test_workload_coefficient_sources():
+    from dataclasses import replace
+    w = wl.WORKLOADS["pro-diffusion"]
+    assert w.coef == "ddim" and w.velocity == "eps" and w.vel_dtype == "fp32"
+    c = [w.step_coef(s) for s in range(w.n_steps)]
+    assert all(cx > 1.0 and cv < 0.0 for cx, cv, _ in c) and c[-1][2] == 0.0 and all(ns > 0 for _, _, ns in c[:-1])
+    p_x, p_v = w.preview_coef(30)
+    assert p_x > 1.0 and p_v < 0.0
+    a, b = wl.eps_mix(w, 30)
+    assert abs(a * a + b * b - 1.0) < 1e-12          # (sigma_t, alpha_t) of a variance-preserving schedule
+    x = torch.randn(5, w.elems)
+    z = wl.normal_noise(wl.scaled(w, n_groups=1), 3, 5)
+    v = wl.eps_velocity(x, z, a, b, "fp32")
+    torch.testing.assert_close(v, a * x + b * z, rtol=1e-6, atol=1e-7)
+    assert wl.eps_velocity(x, z, a, b, "bf16").dtype == torch.bfloat16
+    for coef in ("rf-drift", "rf-sde", "vp-em"):
+        wc = replace(wl.WORKLOADS["sd15"], coef=coef)
+        assert len(wc.step_coef(3)) == 3 and len(wc.preview_coef(3)) == 2
+    assert wl.WORKLOADS["large"].step_coef(5) == (1.0, 1.0 / 28, 0.7 * (1.0 / 28) ** 0.5)
