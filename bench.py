@@ -782,7 +782,7 @@ def run_e2e(B, wl, w, wr, rank, dist, dev, args):
         ids = torch.empty(w.n_groups * K, dtype=torch.int32).pin_memory()
     except Exception as e:            # out of host or device memory
         ok, why = 0.0, f"{type(e).__name__}: {e}"[:200]
-    if -sharding.max_over_ranks(-ok, dist, dev) < 1.0:
+    if not sharding.all_ranks_ok(ok == 1.0, dist, dev):
         return {"value": None, "unit": UNIT, "unavailable": why or "another rank could not allocate its buffers"}
     coefs = [w.step_coef(s) for s in range(w.n_steps)]
     pcoefs = [w.preview_coef(s) for s, _ in w.stages]

@@ -33,6 +33,13 @@ def max_over_ranks(value: float, dist=None, device=None) -> float:
     return float(t.item())
 
 
+def all_ranks_ok(ok: bool, dist=None, device=None) -> bool:
+    """True only if every rank passes True: lets all ranks take the same branch after a step that
+    may fail on some of them (e.g. pinning tens of GB of host memory), so that none is left alone
+    in a later collective."""
+    return max_over_ranks(0.0 if ok else 1.0, dist, device) == 0.0
+
+
 def all_gather_groups(t, dist=None, group=None):
     """Concatenates a per-group (or per-trajectory) tensor over ranks in rank order, i.e. in global
     group order for contiguous shards.  Shards may differ in their first dimension (group_shard

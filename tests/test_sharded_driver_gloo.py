@@ -71,6 +71,10 @@ def _worker(rank, world, port, total, out_dir):
         res = sr.gather(out)
         slowest = sr.max_over_ranks(5.0 + rank)
         assert slowest == 5.0 + world - 1
+        # one rank failing a local step makes every rank skip what follows, together
+        from paper_2512_15347_b200 import sharding
+        assert sharding.all_ranks_ok(True, dist) is True
+        assert sharding.all_ranks_ok(rank != world - 1, dist) is False
         np.savez(os.path.join(out_dir, f"rank{rank}.npz"), adv=res.adv.numpy(), rewards=res.rewards.numpy(),
                  mean=res.mean.numpy(), std=res.std.numpy(), ids=res.traj_id.numpy(),
                  shards=np.array(res.shards))
