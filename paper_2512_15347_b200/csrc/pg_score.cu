@@ -58,7 +58,8 @@ constexpr int kScoreUnroll = 4;   // quads per thread and iteration (loads of th
 // The bf16-prediction variants that also write the preview are held to 64 registers (four CTAs per SM, like the
 // scoring-only variants): at the 69 - 70 registers the compiler would otherwise take, three CTAs
 // fit and the bf16-emitting pass measured 6.47 instead of 6.82 TB/s on 2048 rows of 262144.
-template <typename VelT, bool kUseVel, int kEmit>
+// kReduce = false: emission only (pg_preview): the same streaming loop without the row reduction.
+template <typename VelT, bool kUseVel, int kEmit, bool kReduce = true>
 __global__ void __launch_bounds__(kRowThreads, (kEmit != kEmitNone && sizeof(VelT) == 2) ? 4 : 0)
 score_kernel(const __grid_constant__ ScoreParams p) {
   using Raw = typename VelRaw<VelT>::type;
@@ -105,7 +106,7 @@ score_kernel(const __grid_constant__ ScoreParams p) {
           h.z = fmaf(p.p_v, vf.z, h.z);
           h.w = fmaf(p.p_v, vf.w, h.w);
         }
-        acc += (h.x + h.y) + (h.z + h.w);
+        if (kReduce) acc += (h.x + h.y) + (h.z + h.w);
         if (kEmit) store_preview(prev, (size_t)qq, h);
       }
     }
@@ -114,6 +115,7 @@ score_kernel(const __grid_constant__ ScoreParams p) {
     q = nq;
   }
 
+  if (!kReduce) return;
   acc = warp_sum(acc);
   finish_row(acc, row, chunk, p.chunks, p.partials, p.tickets,
              [&](double sum) { p.scores_out[row] = (float)(sum * p.inv_d); });
@@ -165,58 +167,33 @@ int launch_score(int n_rows, int elems, int vel_dtype, const float* x, const voi
 
 // ---------------------------------------------------------------- preview emission only
 
-
 // x_hat = p_x x + p_v v written in fp32 or bf16 (for a decoder that follows); no reduction.
-template <typename VelT, typename OutT>
-__global__ void __launch_bounds__(kRowThreads)
-preview_kernel(const float* __restrict__ x, const void* __restrict__ vel_v, OutT* __restrict__ out,
-               long long total_quads, float p_x, float p_v) {
-  using Raw = typename VelRaw<VelT>::type;
-  const Raw* vel = reinterpret_cast<const Raw*>(vel_v);
-  constexpr int kU = 4;
-  const long long stride = (long long)gridDim.x * kRowThreads * kU;
-  for (long long q0 = (long long)blockIdx.x * kRowThreads * kU + threadIdx.x; q0 < total_quads; q0 += stride) {
-    float4 xv[kU];
-    Raw vv[kU];
-#pragma unroll
-    for (int u = 0; u < kU; ++u) {
-      const long long q = q0 + u * kRowThreads;
-      if (q < total_quads) {
-        xv[u] = __ldcs(reinterpret_cast<const float4*>(x) + q);
-        vv[u] = __ldcs(vel + q);
-      }
-    }
-#pragma unroll
-    for (int u = 0; u < kU; ++u) {
-      const long long q = q0 + u * kRowThreads;
-      if (q < total_quads) {
-        const float4 vf = unpack_vel(vv[u]);
-        float4 h;
-        h.x = fmaf(p_v, vf.x, p_x * xv[u].x);
-        h.y = fmaf(p_v, vf.y, p_x * xv[u].y);
-        h.z = fmaf(p_v, vf.z, p_x * xv[u].z);
-        h.w = fmaf(p_v, vf.w, p_x * xv[u].w);
-        store_preview(out, (size_t)q, h);
-      }
-    }
-  }
-}
-
 int launch_preview(int n_rows, int elems, int vel_dtype, const float* x, const void* vel, double p_x,
                    double p_v, void* out, int out_bf16, cudaStream_t stream) {
-  const long long total = (long long)n_rows * (elems / 4);
-  if (total == 0) return PG_OK;
-  const long long per_cta = (long long)kRowThreads * 4 * 4;          // 16 quads per thread
-  long long ctas = (total + per_cta - 1) / per_cta;
-  if (ctas > 148LL * 64) ctas = 148LL * 64;
-  const dim3 grid((unsigned)ctas), block(kRowThreads);
-  const float px = (float)p_x, pv = (float)p_v;
+  if (n_rows == 0) return PG_OK;
+  const RowGeometry geo = row_geometry(n_rows, elems);
+  ScoreParams p;
+  p.x = x;
+  p.vel = vel;
+  p.scores_out = nullptr;
+  p.preview_out = out;
+  p.partials = nullptr;
+  p.tickets = nullptr;
+  p.quads_per_row = elems / 4;
+  p.chunk_quads = geo.chunk_quads;
+  p.chunks = geo.chunks;
+  p.p_x = (float)p_x;
+  p.p_v = (float)p_v;
+  p.inv_d = 0.0;
+  const long long blocks = (long long)n_rows * geo.chunks;
+  if (blocks > 0x7FFFFFFFLL) return PG_EINVAL;
+  const dim3 grid((unsigned)blocks), block(kRowThreads);
   if (vel_dtype == PG_VEL_BF16) {
-    if (out_bf16) preview_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, block, 0, stream>>>(x, vel, (__nv_bfloat16*)out, total, px, pv);
-    else          preview_kernel<__nv_bfloat16, float><<<grid, block, 0, stream>>>(x, vel, (float*)out, total, px, pv);
+    if (out_bf16) score_kernel<__nv_bfloat16, true, kEmitBf16, false><<<grid, block, 0, stream>>>(p);
+    else          score_kernel<__nv_bfloat16, true, kEmitF32, false><<<grid, block, 0, stream>>>(p);
   } else {
-    if (out_bf16) preview_kernel<float, __nv_bfloat16><<<grid, block, 0, stream>>>(x, vel, (__nv_bfloat16*)out, total, px, pv);
-    else          preview_kernel<float, float><<<grid, block, 0, stream>>>(x, vel, (float*)out, total, px, pv);
+    if (out_bf16) score_kernel<float, true, kEmitBf16, false><<<grid, block, 0, stream>>>(p);
+    else          score_kernel<float, true, kEmitF32, false><<<grid, block, 0, stream>>>(p);
   }
   PG_LAUNCH_CHECK();
   return PG_OK;
