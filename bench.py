@@ -203,7 +203,7 @@ def run_reference(args):
         return 0
     import oracle
     from paper_2512_15347_b200 import workloads as wl
-    w = wl.WORKLOADS[args.workload]
+    w = wl.load_workload(args.config) if args.config else wl.WORKLOADS[args.workload]
     small = OracleSample(w, 1)
     t1 = min([small.run() for _ in range(max(args.warmup, 1))])
     # bounded sample: as many groups (up to ORACLE_GROUPS) as keep the timed steps near two minutes
@@ -429,7 +429,7 @@ def run_ours(args):
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
-    w = wl.WORKLOADS[args.workload]
+    w = wl.load_workload(args.config) if args.config else wl.WORKLOADS[args.workload]
     if args.groups:
         w = wl.scaled(w, n_groups=args.groups, name=f"{w.name}[{args.groups} groups]")
 
@@ -442,7 +442,7 @@ def run_ours(args):
         cpu_base = {"value": sample.sw.traj_steps / sec, "unit": UNIT, "cores": oracle.num_threads(),
                     "cpu_model": cpu_model(), "kind": "oracle", "sample": sample.desc + f"; best of 2 runs, {sec:.1f} s each"}
         del sample
-        if args.workload == "large" and not args.groups and not args.no_others:
+        if w.name == "large" and not args.groups and not args.no_others:
             for name, groups in OTHER_WORKLOADS:
                 ow = wl.WORKLOADS[name]
                 sm = OracleSample(ow, min(groups, ow.n_groups))
@@ -700,7 +700,7 @@ def run_ours(args):
 
     # the three smaller workloads, same driver (secondary lines; the bench line is the large one)
     others = None
-    if rank == 0 and world == 1 and args.workload == "large" and not args.groups and not args.no_others:
+    if rank == 0 and world == 1 and w.name == "large" and not args.groups and not args.no_others:
         others = {}
         for name, _ in OTHER_WORKLOADS:
             others[name] = _other_workload(name, dev, max(5, min(args.steps, 20)), peak)
@@ -852,6 +852,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="large", choices=["large", "sd3", "sd15", "tiny", "pro-standard", "pro-flash", "pro-diffusion"])
+    ap.add_argument("--config", default="", help="JSON workload file (see paper_2512_15347_b200/configs/) instead of --workload")
     ap.add_argument("--groups", type=int, default=0,
                     help="prompt groups per GPU (default: the workload's own; smaller for profiling)")
     ap.add_argument("--no-e2e", action="store_true")

@@ -13,6 +13,7 @@ settings of Section 6.1).
 """
 from __future__ import annotations
 
+import dataclasses
 import functools
 import math
 from dataclasses import dataclass
@@ -152,6 +153,33 @@ WORKLOADS: Dict[str, Workload] = {
     "pro-diffusion": Workload("pro-diffusion", 16, 48, ((30, 32), (40, 8)), 50, 4 * 64 * 64, 4, "fp32",
                               13, "eps", "preview", coef="ddim", eta=1.0),
 }
+
+def workload_to_dict(w: Workload) -> dict:
+    d = dataclasses.asdict(w)
+    d["stages"] = [list(st) for st in w.stages]
+    return d
+
+
+def workload_from_dict(d: dict) -> Workload:
+    """A workload from its JSON form (the files under configs/ mirror the built-in ones; a caller
+    can describe its own batch shape and schedule the same way)."""
+    d = dict(d)
+    d["stages"] = tuple((int(s), int(k)) for s, k in d.get("stages", ()))
+    unknown = set(d) - {f.name for f in dataclasses.fields(Workload)}
+    if unknown:
+        raise ValueError(f"unknown workload fields: {sorted(unknown)}")
+    w = Workload(**d)
+    sch.validate_stages(w.n_expand, w.n_steps, w.stages)
+    if w.elems % 4 or w.elems < 4 or w.vel_dtype not in ("fp32", "bf16"):
+        raise ValueError("elems must be a positive multiple of 4 and vel_dtype fp32 or bf16")
+    return w
+
+
+def load_workload(path: str) -> Workload:
+    import json
+    with open(path) as f:
+        return workload_from_dict(json.load(f))
+
 
 # OVF selection microbenchmark: 4096 groups x 256 scores, keep 32.
 OVF_MICRO = dict(n_groups=4096, n=256, k=32, seed=4)

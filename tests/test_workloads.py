@@ -77,3 +77,26 @@ def test_workload_coefficient_sources():
         wc = replace(wl.WORKLOADS["sd15"], coef=coef)
         assert len(wc.step_coef(3)) == 3 and len(wc.preview_coef(3)) == 2
     assert wl.WORKLOADS["large"].step_coef(5) == (1.0, 1.0 / 28, 0.7 * (1.0 / 28) ** 0.5)
+
+
+def test_config_files_mirror_the_built_in_workloads(tmp_path):
+    import glob, json, os
+    here = os.path.join(os.path.dirname(os.path.dirname(os.path.abspath(__file__))), "paper_2512_15347_b200", "configs")
+    files = sorted(glob.glob(os.path.join(here, "*.json")))
+    names = {os.path.splitext(os.path.basename(f))[0] for f in files}
+    assert names == set(wl.WORKLOADS) | {"ovf_micro"}
+    for name, w in wl.WORKLOADS.items():
+        assert wl.load_workload(os.path.join(here, name + ".json")) == w
+    micro = json.load(open(os.path.join(here, "ovf_micro.json")))
+    assert {k: micro[k] for k in wl.OVF_MICRO} == wl.OVF_MICRO
+    bad = wl.workload_to_dict(wl.WORKLOADS["sd15"])
+    bad["stages"] = [[4, 30]]
+    p = tmp_path / "bad.json"
+    p.write_text(json.dumps(bad))
+    import pytest
+    with pytest.raises(ValueError):
+        wl.load_workload(str(p))
+    bad = wl.workload_to_dict(wl.WORKLOADS["sd15"])
+    bad["colour"] = "red"
+    with pytest.raises(ValueError):
+        wl.workload_from_dict(bad)
