@@ -67,26 +67,30 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
 // Box-Muller on two generator words (24-bit uniforms):
 //   u1 = ((r0 >> 8) + 1) * 2^-24 in (0, 1],  u2 = (r1 >> 8) * 2^-24 in [0, 1)
 //   normals  a = sqrt(-2 ln u1) cos(2 pi u2),  b = sqrt(-2 ln u1) sin(2 pi u2)
-// Returned in factored form: radius = sqrt(-2 ln u1) and (c, s) = (cos, sin)(2 pi u2 - pi), so
-// that a = -radius * c and b = -radius * s (half-turn shift: the hardware sine is evaluated on
-// [-pi, pi), its most accurate range); the return value is -2 ln u1 = a^2 + b^2.
+// Returned in factored and scaled form: with neg_scale2 = -2 ln 2 * scale^2 the outputs are
+// radius = scale * sqrt(-2 ln u1) and (c, s) = (cos, sin)(2 pi u2 - pi), so that scale * a =
+// -radius * c and scale * b = -radius * s (half-turn shift: the hardware sine is evaluated on
+// [-pi, pi), its most accurate range); the return value is log2(u1) <= 0, i.e. a^2 + b^2 =
+// -2 ln 2 * (return value).  Keeping the logarithm in base 2 until the square root saves a
+// multiplication per pair: the caller sums the returned values and applies -2 ln 2 once.
 // The logarithm uses the hardware log2 except close to u1 = 1, where its absolute error would
-// dominate the small radius: there -2 ln(1 - w) is summed as a short series in w = 1 - u1 (exact
+// dominate the small radius: there log2(1 - w) is summed as a short series in w = 1 - u1 (exact
 // in fp32; truncation below 2e-8 relative for w < 2^-6).
-__device__ __forceinline__ float box_muller(uint32_t r0, uint32_t r1, float& radius, float& c, float& s) {
+constexpr float kTwoLn2 = 1.3862943611198906f;
+__device__ __forceinline__ float box_muller(uint32_t r0, uint32_t r1, float neg_scale2, float& radius, float& c,
+                                            float& s) {
   const float k1 = (float)(r0 >> 8);
   const float u1 = fmaf(k1, 5.9604644775390625e-8f, 5.9604644775390625e-8f);
   float lg;                                                     // u1 >= 2^-24: never subnormal
   asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(lg) : "f"(u1));
-  float neg2ln = -1.3862943611198906f * lg;                     // -2 ln(u1) = -2 ln2 * log2(u1)
   const float w = 1.0f - u1;                                     // exact (24-bit grid)
-  // -2 ln(1 - w) = 2w + w^2 + (2/3) w^3 + (1/2) w^4 + ...
-  float ser = fmaf(w, 0.5f, 0.66666666666666667f);
-  ser = fmaf(ser, w, 1.0f);
-  ser = fmaf(ser, w, 2.0f);
+  // log2(1 - w) = -(w + w^2/2 + w^3/3 + w^4/4 + ...) / ln 2
+  float ser = fmaf(w, -0.36067376022224085f, -0.48089834696298783f);
+  ser = fmaf(ser, w, -0.7213475204444817f);
+  ser = fmaf(ser, w, -1.4426950408889634f);
   ser *= w;
-  neg2ln = (w < 0.015625f) ? ser : neg2ln;
-  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(radius) : "f"(neg2ln));
+  lg = (w < 0.015625f) ? ser : lg;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(radius) : "f"(lg * neg_scale2));
   const float turn = fmaf((float)(r1 >> 8), 5.9604644775390625e-8f, -0.5f);  // u2 - 1/2, exact
   // The cosine is taken as a sine: cos t = sin(pi/2 - |t|), i.e. the sine at 1/4 - |turn| turns
   // (an exact difference on the 24-bit grid, and an argument in [-pi/2, pi/2]).  The hardware
@@ -98,16 +102,15 @@ __device__ __forceinline__ float box_muller(uint32_t r0, uint32_t r1, float& rad
   const float angle_c = 6.283185307179586f * (0.25f - fabsf(turn));
   asm("sin.approx.ftz.f32 %0, %1;" : "=f"(s) : "f"(angle));
   asm("sin.approx.ftz.f32 %0, %1;" : "=f"(c) : "f"(angle_c));
-  return neg2ln;
+  return lg;
 }
 
 // The two normals themselves.
-__device__ __forceinline__ float normal_pair(uint32_t r0, uint32_t r1, float& a, float& b) {
+__device__ __forceinline__ void normal_pair(uint32_t r0, uint32_t r1, float& a, float& b) {
   float radius, c, s;
-  const float neg2ln = box_muller(r0, r1, radius, c, s);
+  box_muller(r0, r1, -kTwoLn2, radius, c, s);
   a = -radius * c;
   b = -radius * s;
-  return neg2ln;
 }
 
 // Bounded wait on an mbarrier in shared memory (`bar` = shared-space address) for the phase of

@@ -5,7 +5,7 @@
 // current pair is computed (full chunks alternate between two register sets without bounds
 // checks); the noise is generated in registers (one Philox block per 4 elements); x' is written
 // once.  Sum of squared noise: for a Box-Muller pair a^2 + b^2 equals -2 ln u1, so the radius
-// term is accumulated directly.  The per-trajectory sum is reduced thread -> warp (shuffle) ->
+// term (as log2 u1, scaled once per thread) is accumulated directly.  The per-trajectory sum is reduced thread -> warp (shuffle) ->
 // CTA (shared memory) -> trajectory (fixed-slot partials finished by the last-arriving CTA,
 // without waiting), so the result does not depend on scheduling.
 #include "pg_common.cuh"
@@ -26,8 +26,10 @@ struct StepParams {
   int quads_per_row;      // d / 4
   int chunk_quads;        // quads per CTA
   int chunks;             // CTAs per row
+  int chunk_shift;        // log2(chunks) when chunks is a power of two, else -1
   uint32_t step;
-  float c_x, c_v, neg_noise_std;
+  float c_x, c_v;
+  float neg_scale2;       // -2 ln 2 * noise_std^2: log2(u1) times this is (noise_std * radius)^2
   double logp_const;      // d/2 * ln(2 pi noise_std^2)
   double logp_scale;      // 1 or 1/d
   PhiloxKeys rk;
@@ -87,16 +89,14 @@ __device__ __forceinline__ void step_quad(const StepParams& p, uint32_t traj, in
   }
   if (kNoise) {
     const uint4 r = philox4x32_10((uint32_t)q, p.step, traj, 0u, p.rk);
-    // noise_std * xi = (-noise_std * radius) * (cos, sin): the scale is applied once per pair
+    // noise_std * xi = -(noise_std * radius) * (cos, sin): the scale enters under the square root
     float ra, ca, sa, rb, cb, sb;
-    acc += box_muller(r.x, r.y, ra, ca, sa);
-    acc += box_muller(r.z, r.w, rb, cb, sb);
-    ra *= p.neg_noise_std;
-    rb *= p.neg_noise_std;
-    m.x = fmaf(ra, ca, m.x);
-    m.y = fmaf(ra, sa, m.y);
-    m.z = fmaf(rb, cb, m.z);
-    m.w = fmaf(rb, sb, m.w);
+    acc += box_muller(r.x, r.y, p.neg_scale2, ra, ca, sa);       // acc collects log2(u1) <= 0
+    acc += box_muller(r.z, r.w, p.neg_scale2, rb, cb, sb);
+    m.x = fmaf(-ra, ca, m.x);
+    m.y = fmaf(-ra, sa, m.y);
+    m.z = fmaf(-rb, cb, m.z);
+    m.w = fmaf(-rb, sb, m.w);
   }
   __stcs(xout + q, m);
 }
@@ -106,7 +106,8 @@ template <typename VelT, bool kNoise, bool kUnitCx>
 __global__ void __launch_bounds__(kRowThreads, StepMinCtas<VelT, kNoise>::value)
 step_kernel(const __grid_constant__ StepParams p) {
   using VReg = typename VelReg<VelT>::type;
-  const int row = blockIdx.x / p.chunks;
+  // chunks per row is a power of two for the usual latent sizes: a shift instead of a division
+  const int row = p.chunk_shift >= 0 ? (int)(blockIdx.x >> p.chunk_shift) : (int)(blockIdx.x / p.chunks);
   const int chunk = blockIdx.x - row * p.chunks;
   int src = p.src_rows ? p.src_rows[row] : row;
   if ((unsigned int)src >= (unsigned int)p.rows_in) {
@@ -188,7 +189,7 @@ step_kernel(const __grid_constant__ StepParams p) {
     if (chunk == 0 && threadIdx.x == 0) p.logp_out[row] = 0.f;
     return;
   }
-  acc = warp_sum(acc);
+  acc = warp_sum(acc * -kTwoLn2);               // sum of squared noise = -2 ln 2 * sum of log2(u1)
   float* logp_out = p.logp_out;
   const double logp_const = p.logp_const, logp_scale = p.logp_scale;
   finish_row(acc, row, chunk, p.chunks, p.partials, p.tickets,
@@ -226,10 +227,13 @@ int launch_step(int n_rows, int elems, int vel_dtype, const float* x_in, const v
   p.quads_per_row = elems / 4;
   p.chunk_quads = geo.chunk_quads;
   p.chunks = geo.chunks;
+  p.chunk_shift = -1;
+  for (int b = 0; b < 31; ++b)
+    if (geo.chunks == (1 << b)) p.chunk_shift = b;
   p.step = (uint32_t)step;
   p.c_x = (float)c_x;
   p.c_v = (float)c_v;
-  p.neg_noise_std = -(float)noise_std;
+  p.neg_scale2 = (float)(-1.3862943611198906 * noise_std * noise_std);
   const double two_pi = 6.283185307179586476925286766559;
   p.logp_const = noise_std > 0.0 ? 0.5 * (double)elems * log(two_pi * noise_std * noise_std) : 0.0;
   p.logp_scale = logp_mean ? 1.0 / (double)elems : 1.0;
