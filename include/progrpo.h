@@ -153,6 +153,17 @@ int pg_step(pg_rollout *h, int32_t step, const pg_step_coef *coef, const float *
             const void *vel, const int32_t *src_rows, float *x_out, float *logp_out, void *stream);
 
 /*
+ * pg_step that also returns the mean of every updated latent: reward_out[i] = mean_e(x_out[i][e]),
+ * [n_active] fp32 - the stand-in for the final reward R(x_T, c) of Eq. "advK" when `step` is the last
+ * step (the value pg_score(p_x = 1, p_v = 0) would compute from x_out, up to the order of the fp32
+ * additions), reduced from the registers that hold x' so that the final latents are not read again.
+ * Everything else as pg_step; valid at any step.
+ */
+int pg_step_reward(pg_rollout *h, int32_t step, const pg_step_coef *coef, const float *x_in,
+                   const void *vel, const int32_t *src_rows, float *x_out, float *logp_out,
+                   float *reward_out, void *stream);
+
+/*
  * Latent score at a pruning checkpoint (Eq. "ode_lookahead_method", Eq.
  * "proxy_reward_method").  The preview x_hat = p_x * x + p_v * vel is reduced
  * to the stand-in proxy reward r = mean_e(x_hat_e) for each of the n_active

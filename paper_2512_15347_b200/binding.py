@@ -73,6 +73,7 @@ def lib() -> ctypes.CDLL:
     L.pg_rollout_restore.argtypes = [vp, i32, i32, vp, vp]
     L.pg_rollout_status.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
     L.pg_step.argtypes = [vp, i32, ctypes.POINTER(StepCoef), vp, vp, vp, vp, vp, vp]
+    L.pg_step_reward.argtypes = [vp, i32, ctypes.POINTER(StepCoef), vp, vp, vp, vp, vp, vp, vp]
     L.pg_score.argtypes = [vp, ctypes.POINTER(PreviewCoef), vp, vp, vp, vp, vp]
     L.pg_preview.argtypes = [vp, ctypes.POINTER(PreviewCoef), vp, vp, vp, i32, vp]
     L.pg_score_preview.argtypes = [vp, ctypes.POINTER(PreviewCoef), vp, vp, vp, vp, i32, vp]
@@ -113,7 +114,7 @@ def lib() -> ctypes.CDLL:
                  "pg_step", "pg_score", "pg_prune_ovf", "pg_compact", "pg_advantages",
                  "pg_ovf_select_batched", "pg_rollout_host", "pg_rollout_traj_ids",
                  "pg_philox_raw", "pg_normal_rows", "pg_score_static", "pg_policy_logprob",
-                 "pg_policy_objective", "pg_policy_backward", "pg_prune_uniform", "pg_group_stats", "pg_preview", "pg_rollout_run", "pg_rollout_restore", "pg_score_preview", "pg_rollout_host_on"):
+                 "pg_policy_objective", "pg_policy_backward", "pg_prune_uniform", "pg_group_stats", "pg_preview", "pg_rollout_run", "pg_rollout_restore", "pg_score_preview", "pg_rollout_host_on", "pg_step_reward"):
         getattr(L, name).restype = ctypes.c_int
     _lib = L
     return L
@@ -189,6 +190,14 @@ def step(h: int, step_index: int, coef, x_in, vel, src_rows, x_out, logp_out, st
     c = StepCoef(*coef)
     _check(lib().pg_step(h, step_index, ctypes.byref(c), _p(x_in), _p(vel), _p(src_rows), _p(x_out),
                          _p(logp_out), _stream(stream)), "pg_step")
+
+
+def step_reward(h: int, step_index: int, coef, x_in, vel, src_rows, x_out, logp_out, reward_out,
+                stream=None) -> None:
+    """pg_step that also writes the mean of every updated latent (the final-reward stand-in)."""
+    c = StepCoef(*coef)
+    _check(lib().pg_step_reward(h, step_index, ctypes.byref(c), _p(x_in), _p(vel), _p(src_rows), _p(x_out),
+                                _p(logp_out), _p(reward_out), _stream(stream)), "pg_step_reward")
 
 
 def score(h: int, coef, x, vel, scores_out, preview_out=None, stream=None) -> None:

@@ -267,7 +267,7 @@ int launch_step(int n_rows, int elems, int vel_dtype, const float* x_in, const v
                 const int32_t* src_rows, const int32_t* traj_id, float* x_out, float* logp_out,
                 uint64_t seed, int32_t step, double c_x, double c_v, double noise_std,
                 int logp_mean, RowScratch scratch, cudaStream_t stream, int rows_in = 0,
-                int32_t* status = nullptr);
+                int32_t* status = nullptr, float* xmean_out = nullptr);
 
 int launch_score(int n_rows, int elems, int vel_dtype, const float* x, const void* vel,
                  double p_x, double p_v, float* scores_out, void* preview_out, int preview_bf16,

@@ -229,8 +229,11 @@ int pg_rollout_status(pg_rollout* h, int32_t* n_active, int32_t* next_step, int3
   return PG_OK;
 }
 
-int pg_step(pg_rollout* h, int32_t step, const pg_step_coef* coef, const float* x_in,
-            const void* vel, const int32_t* src_rows, float* x_out, float* logp_out, void* stream) {
+}  // extern "C"
+
+static int step_impl(pg_rollout* h, int32_t step, const pg_step_coef* coef, const float* x_in,
+                     const void* vel, const int32_t* src_rows, float* x_out, float* logp_out,
+                     float* xmean_out, void* stream) {
   TraceRange trace_range("pg_step");
   if (!h || !coef || !x_in || !vel || !x_out || !logp_out) return PG_EINVAL;
   if (const int rc_dev = wrong_device(h)) return rc_dev;
@@ -255,9 +258,23 @@ int pg_step(pg_rollout* h, int32_t step, const pg_step_coef* coef, const float* 
                                  h->d_traj[h->traj_cur], x_out, logp_out, h->cfg.seed, step,
                                  coef->c_x, coef->c_v, coef->noise_std, h->cfg.logp_mean, scratch,
                                  (cudaStream_t)stream,
-                                 src_rows ? h->cfg.n_groups * h->k_prev : rows, h->d_status);
+                                 src_rows ? h->cfg.n_groups * h->k_prev : rows, h->d_status, xmean_out);
   if (rc == PG_OK) h->next_step = step + 1;
   return rc;
+}
+
+extern "C" {
+
+int pg_step(pg_rollout* h, int32_t step, const pg_step_coef* coef, const float* x_in,
+            const void* vel, const int32_t* src_rows, float* x_out, float* logp_out, void* stream) {
+  return step_impl(h, step, coef, x_in, vel, src_rows, x_out, logp_out, nullptr, stream);
+}
+
+int pg_step_reward(pg_rollout* h, int32_t step, const pg_step_coef* coef, const float* x_in,
+                   const void* vel, const int32_t* src_rows, float* x_out, float* logp_out,
+                   float* reward_out, void* stream) {
+  if (!reward_out) return PG_EINVAL;
+  return step_impl(h, step, coef, x_in, vel, src_rows, x_out, logp_out, reward_out, stream);
 }
 
 int pg_score_preview(pg_rollout* h, const pg_preview_coef* coef, const float* x, const void* vel,
@@ -647,18 +664,17 @@ int pg_rollout_host_on(pg_rollout* h, const pg_step_coef* step_coef,
       ++stage;
     }
     float* x_out = src ? d_x[cur ^ 1] : d_x[cur];
-    PG_TRY(pg_step(h, s, &step_coef[s], d_x[cur], d_v[b], src, x_out, d_logp + logp_off, compute));
+    if (s == cfg->n_steps - 1 && !final_rewards)      // the last step also reduces the reward stand-in
+      PG_TRY(pg_step_reward(h, s, &step_coef[s], d_x[cur], d_v[b], src, x_out, d_logp + logp_off, d_rewards, compute));
+    else
+      PG_TRY(pg_step(h, s, &step_coef[s], d_x[cur], d_v[b], src, x_out, d_logp + logp_off, compute));
     if (src) cur ^= 1;
     logp_off += (size_t)cfg->n_groups * h->k_cur;
     PG_TRY_CUDA(cudaEventRecord(v_free[b], compute));
   }
   const size_t rows_final = (size_t)cfg->n_groups * h->k_cur;
-  if (final_rewards) {
+  if (final_rewards)
     PG_TRY_CUDA(cudaMemcpyAsync(d_rewards, final_rewards, rows_final * 4, cudaMemcpyHostToDevice, compute));
-  } else {
-    const pg_preview_coef id = {1.0, 0.0};
-    PG_TRY(pg_score(h, &id, d_x[cur], nullptr, d_rewards, nullptr, compute));
-  }
   PG_TRY(pg_advantages(h, d_rewards, d_adv, nullptr, nullptr, compute));
   PG_TRY(pg_rollout_traj_ids(h, d_traj, compute));
   if (x_final) PG_TRY_CUDA(cudaMemcpyAsync(x_final, d_x[cur], rows_final * cfg->elems * 4, cudaMemcpyDeviceToHost, compute));
@@ -772,19 +788,16 @@ int pg_rollout_run(pg_rollout* h, const pg_step_coef* step_coef, const pg_previe
     if (cur < 0) { x_out = d_x[0]; }
     else if (src) { x_out = d_x[cur ^ 1]; }
     else { x_out = d_x[cur]; }
-    rc = pg_step(h, s, &step_coef[s], x_cur, vel_steps[s], src, x_out, d_logp + logp_off, stream);
+    if (s == cfg->n_steps - 1 && !final_rewards)      // the last step also reduces the reward stand-in
+      rc = pg_step_reward(h, s, &step_coef[s], x_cur, vel_steps[s], src, x_out, d_logp + logp_off, d_rewards, stream);
+    else
+      rc = pg_step(h, s, &step_coef[s], x_cur, vel_steps[s], src, x_out, d_logp + logp_off, stream);
     if (rc != PG_OK) return rc;
     if (cur < 0) cur = 0; else if (src) cur ^= 1;
     x_cur = d_x[cur];
     logp_off += (size_t)cfg->n_groups * h->k_cur;
   }
-  const float* rw = final_rewards;
-  if (!rw) {
-    const pg_preview_coef id = {1.0, 0.0};
-    rc = pg_score(h, &id, x_cur, nullptr, d_rewards, nullptr, stream);
-    if (rc != PG_OK) return rc;
-    rw = d_rewards;
-  }
+  const float* rw = final_rewards ? final_rewards : d_rewards;
   rc = pg_advantages(h, rw, d_adv, nullptr, nullptr, stream);
   if (rc != PG_OK) return rc;
   rc = pg_rollout_traj_ids(h, d_traj, stream);

@@ -19,6 +19,7 @@ struct StepParams {
   const int32_t* traj_id;
   float* x_out;
   float* logp_out;
+  float* xmean_out;       // [rows] mean of x_out per row, or null
   float* partials;
   unsigned int* tickets;
   int32_t* status;        // device status word (bit 2: gather index out of range) or null
@@ -32,6 +33,7 @@ struct StepParams {
   float neg_scale2;       // -2 ln 2 * noise_std^2: log2(u1) times this is (noise_std * radius)^2
   double logp_const;      // d/2 * ln(2 pi noise_std^2)
   double logp_scale;      // 1 or 1/d
+  double inv_d;           // 1/d
   PhiloxKeys rk;
 };
 
@@ -63,18 +65,20 @@ template <> struct VelReg<__nv_bfloat16> { using type = VelBf16; };
 #ifndef PG_STEP_MIN_CTAS
 #define PG_STEP_MIN_CTAS 5     // __launch_bounds__ minimum resident CTAs per SM (bf16 prediction)
 #endif
-// fp32 predictions keep twice the prediction registers in flight: one CTA less per SM, no spills
-template <typename VelT, bool kNoise> struct StepMinCtas {
-  static constexpr int value = (sizeof(VelT) == 2 && kNoise) ? PG_STEP_MIN_CTAS : 4;
+// fp32 predictions keep twice the prediction registers in flight, and the variant that also reduces
+// the row means one more accumulator: one CTA less per SM, no spills
+template <typename VelT, bool kNoise, bool kMean> struct StepMinCtas {
+  static constexpr int value = (sizeof(VelT) == 2 && kNoise && !kMean) ? PG_STEP_MIN_CTAS : 4;
 };
 constexpr int kStepUnroll = PG_STEP_UNROLL;
 static_assert(kChunkQuads % (2 * kStepUnroll * kRowThreads) == 0,
               "full chunks must hold an even number of batches");
 
 // One quad: mean of the transition, noise, store, radius-term accumulation.
-template <bool kNoise, bool kUnitCx>
+template <bool kNoise, bool kUnitCx, bool kMean>
 __device__ __forceinline__ void step_quad(const StepParams& p, uint32_t traj, int q, const float4& xv,
-                                          const float4& vv, float4* __restrict__ xout, float& acc) {
+                                          const float4& vv, float4* __restrict__ xout, float& acc,
+                                          float& acc_x) {
   float4 m;
   if (kUnitCx) {
     m.x = fmaf(p.c_v, vv.x, xv.x);
@@ -98,12 +102,15 @@ __device__ __forceinline__ void step_quad(const StepParams& p, uint32_t traj, in
     m.z = fmaf(-rb, cb, m.z);
     m.w = fmaf(-rb, sb, m.w);
   }
+  if (kMean) acc_x += (m.x + m.y) + (m.z + m.w);
   __stcs(xout + q, m);
 }
 
 // kNoise: noise_std > 0.  kUnitCx: c_x == 1 (drift = prediction), one FMA per element less.
-template <typename VelT, bool kNoise, bool kUnitCx>
-__global__ void __launch_bounds__(kRowThreads, StepMinCtas<VelT, kNoise>::value)
+// kMean: also reduce the mean of every updated latent (the stand-in reward of the final latent,
+// taken from the registers that hold x' instead of reading x' back in a pass of its own).
+template <typename VelT, bool kNoise, bool kUnitCx, bool kMean>
+__global__ void __launch_bounds__(kRowThreads, StepMinCtas<VelT, kNoise, kMean>::value)
 step_kernel(const __grid_constant__ StepParams p) {
   using VReg = typename VelReg<VelT>::type;
   // chunks per row is a power of two for the usual latent sizes: a shift instead of a division
@@ -124,7 +131,7 @@ step_kernel(const __grid_constant__ StepParams p) {
   const int q_begin = chunk * p.chunk_quads;
   const int q_end = min(q_begin + p.chunk_quads, p.quads_per_row);
 
-  float acc = 0.f;
+  float acc = 0.f, acc_x = 0.f;
   float4 xv[kStepUnroll], nx[kStepUnroll];
   VReg vv[kStepUnroll], nv[kStepUnroll];
   int q = q_begin + threadIdx.x;
@@ -146,7 +153,7 @@ step_kernel(const __grid_constant__ StepParams p) {
       }
 #pragma unroll
       for (int u = 0; u < kStepUnroll; ++u)
-        step_quad<kNoise, kUnitCx>(p, traj, q + u * kRowThreads, xv[u], vel_f32(vv[u]), xout, acc);
+        step_quad<kNoise, kUnitCx, kMean>(p, traj, q + u * kRowThreads, xv[u], vel_f32(vv[u]), xout, acc, acc_x);
       if (it + 2 < iters) {
 #pragma unroll
         for (int u = 0; u < kStepUnroll; ++u) {
@@ -156,7 +163,7 @@ step_kernel(const __grid_constant__ StepParams p) {
       }
 #pragma unroll
       for (int u = 0; u < kStepUnroll; ++u)
-        step_quad<kNoise, kUnitCx>(p, traj, q + kStride + u * kRowThreads, nx[u], vel_f32(nv[u]), xout, acc);
+        step_quad<kNoise, kUnitCx, kMean>(p, traj, q + kStride + u * kRowThreads, nx[u], vel_f32(nv[u]), xout, acc, acc_x);
       q += 2 * kStride;
     }
     q = q_end;
@@ -178,39 +185,50 @@ step_kernel(const __grid_constant__ StepParams p) {
 #pragma unroll
     for (int u = 0; u < kStepUnroll; ++u) {
       const int qq = q + u * kRowThreads;
-      if (qq < q_end) step_quad<kNoise, kUnitCx>(p, traj, qq, xv[u], vel_f32(vv[u]), xout, acc);
+      if (qq < q_end) step_quad<kNoise, kUnitCx, kMean>(p, traj, qq, xv[u], vel_f32(vv[u]), xout, acc, acc_x);
     }
 #pragma unroll
     for (int u = 0; u < kStepUnroll; ++u) { xv[u] = nx[u]; vv[u] = nv[u]; }
     q = nq;
   }
 
-  if (!kNoise) {
+  if (!kNoise && !kMean) {
     if (chunk == 0 && threadIdx.x == 0) p.logp_out[row] = 0.f;
     return;
   }
   acc = warp_sum(acc * -kTwoLn2);               // sum of squared noise = -2 ln 2 * sum of log2(u1)
   float* logp_out = p.logp_out;
   const double logp_const = p.logp_const, logp_scale = p.logp_scale;
-  finish_row(acc, row, chunk, p.chunks, p.partials, p.tickets,
-             [=](double sum) { logp_out[row] = (float)((-0.5 * sum - logp_const) * logp_scale); });
+  if (kMean) {
+    const float totals[2] = {acc, warp_sum(acc_x)};
+    float* xmean_out = p.xmean_out;
+    const double inv_d = p.inv_d;
+    finish_row_n<2>(totals, row, chunk, p.chunks, p.partials, p.tickets, [=](const double (&sum)[2]) {
+      logp_out[row] = kNoise ? (float)((-0.5 * sum[0] - logp_const) * logp_scale) : 0.f;
+      xmean_out[row] = (float)(sum[1] * inv_d);
+    });
+  } else {
+    finish_row(acc, row, chunk, p.chunks, p.partials, p.tickets,
+               [=](double sum) { logp_out[row] = (float)((-0.5 * sum - logp_const) * logp_scale); });
+  }
 }
 
-template <typename VelT>
+template <typename VelT, bool kMean>
 static void dispatch_step(const StepParams& p, bool noise, bool unit_cx, dim3 grid, cudaStream_t st) {
   const dim3 block(kRowThreads);
   if (noise) {
-    if (unit_cx) step_kernel<VelT, true, true><<<grid, block, 0, st>>>(p);
-    else         step_kernel<VelT, true, false><<<grid, block, 0, st>>>(p);
+    if (unit_cx) step_kernel<VelT, true, true, kMean><<<grid, block, 0, st>>>(p);
+    else         step_kernel<VelT, true, false, kMean><<<grid, block, 0, st>>>(p);
   } else {
-    step_kernel<VelT, false, false><<<grid, block, 0, st>>>(p);
+    step_kernel<VelT, false, false, kMean><<<grid, block, 0, st>>>(p);
   }
 }
 
 int launch_step(int n_rows, int elems, int vel_dtype, const float* x_in, const void* vel,
                 const int32_t* src_rows, const int32_t* traj_id, float* x_out, float* logp_out,
                 uint64_t seed, int32_t step, double c_x, double c_v, double noise_std,
-                int logp_mean, RowScratch scratch, cudaStream_t stream, int rows_in, int32_t* status) {
+                int logp_mean, RowScratch scratch, cudaStream_t stream, int rows_in, int32_t* status,
+                float* xmean_out) {
   if (n_rows == 0) return PG_OK;
   const RowGeometry geo = row_geometry(n_rows, elems);
   StepParams p;
@@ -222,6 +240,8 @@ int launch_step(int n_rows, int elems, int vel_dtype, const float* x_in, const v
   p.traj_id = traj_id;
   p.x_out = x_out;
   p.logp_out = logp_out;
+  p.xmean_out = xmean_out;
+  p.inv_d = 1.0 / (double)elems;
   p.partials = scratch.partials;
   p.tickets = scratch.tickets;
   p.quads_per_row = elems / 4;
@@ -242,8 +262,14 @@ int launch_step(int n_rows, int elems, int vel_dtype, const float* x_in, const v
   if (blocks > 0x7FFFFFFFLL) return PG_EINVAL;
   const dim3 grid((unsigned)blocks);
   const bool noise = noise_std > 0.0;
-  if (vel_dtype == PG_VEL_BF16) dispatch_step<__nv_bfloat16>(p, noise, p.c_x == 1.0f, grid, stream);
-  else                          dispatch_step<float>(p, noise, p.c_x == 1.0f, grid, stream);
+  const bool unit_cx = p.c_x == 1.0f;
+  if (vel_dtype == PG_VEL_BF16) {
+    if (xmean_out) dispatch_step<__nv_bfloat16, true>(p, noise, unit_cx, grid, stream);
+    else           dispatch_step<__nv_bfloat16, false>(p, noise, unit_cx, grid, stream);
+  } else {
+    if (xmean_out) dispatch_step<float, true>(p, noise, unit_cx, grid, stream);
+    else           dispatch_step<float, false>(p, noise, unit_cx, grid, stream);
+  }
   PG_LAUNCH_CHECK();
   return PG_OK;
 }

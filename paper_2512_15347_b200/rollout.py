@@ -164,7 +164,13 @@ class Rollout:
                 dst = self.x[self.cur ^ 1] if x_cur is self.x[self.cur] else self.x[self.cur]
             else:
                 dst = x_cur                                 # in place
-            self._timed("step", rows, lambda: B.step(self.h, s, step_coef(s), x_cur, vel, src, dst, lp))
+            if s == self.T - 1 and final_rewards is None:
+                # the last step also reduces the stand-in reward (mean of x_T) from its registers
+                rw_fused = self.rewards[:rows]
+                self._timed("step", rows, lambda: B.step_reward(self.h, s, step_coef(s), x_cur, vel, src, dst,
+                                                                lp, rw_fused))
+            else:
+                self._timed("step", rows, lambda: B.step(self.h, s, step_coef(s), x_cur, vel, src, dst, lp))
             if dst is not x_cur:
                 if x_cur is not x0:
                     self.cur ^= 1
@@ -175,8 +181,7 @@ class Rollout:
         if final_rewards is not None:
             rw = final_rewards()
         else:
-            rw = self.rewards[:rows]
-            self._timed("reward", rows, lambda: B.score(self.h, (1.0, 0.0), x_cur, None, rw))
+            rw = self.rewards[:rows]                      # written by the last step
         self._timed("advantages", rows, lambda: B.advantages(self.h, rw, self.adv, self.mean, self.std))
         ids = torch.empty(rows, device=self.dev, dtype=torch.int32)
         B.rollout_traj_ids(self.h, ids)

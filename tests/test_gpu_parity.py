@@ -92,6 +92,41 @@ def test_step_matches_oracle(B, bf16, d):
         B.rollout_destroy(h)
 
 
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("d", [4, 1000, 3 * 8192 + 20, 262144])
+def test_step_with_fused_reward_matches_oracle(B, bf16, d):
+    """pg_step_reward: latents and log-probs are pg_step's bit for bit; the reward is the mean of the
+    updated latent (the oracle's final-reward stand-in) within the score tolerance; also for the
+    deterministic step and with a gather."""
+    n_groups, n0 = 3, 4
+    n = n_groups * n0
+    rng = np.random.default_rng(3 * d + bf16)
+    x = rng.standard_normal((n, d)).astype(np.float32) + 0.1
+    vt = torch.from_numpy(rng.standard_normal((n, d)).astype(np.float32))
+    vt = vt.to(torch.bfloat16) if bf16 else vt
+    v = wl.as_numpy_velocity(vt)
+    x_dev, v_dev = U.to_dev(x), U.vel_to_dev(v)
+    for coef in ((1.0, 0.05, 0.15), (1.1, -0.2, 0.3), (0.5, 0.25, 0.0)):
+        outs = []
+        for fused in (False, True):
+            h, _ = _handle(B, n_groups, n0, d, seed=21, bf16=bf16)
+            x_out = torch.empty_like(x_dev)
+            lp = torch.empty(n, device="cuda")
+            rw = torch.full((n,), float("nan"), device="cuda")
+            if fused:
+                B.step_reward(h, 0, coef, x_dev, v_dev, None, x_out, lp, rw)
+            else:
+                B.step(h, 0, coef, x_dev, v_dev, None, x_out, lp)
+            torch.cuda.synchronize()
+            B.rollout_destroy(h)
+            outs.append((x_out, lp, rw))
+        assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+        ref_x, ref_lp = oracle.step(x, v, np.arange(n, dtype=np.int32), 21, 0, *coef)
+        assert U.latent_err(outs[1][0].cpu().numpy(), ref_x) <= U.LATENT_TOL
+        ref_rw = ref_x.astype(np.float64).mean(axis=1)
+        assert np.abs(outs[1][2].cpu().numpy() - ref_rw).max() <= U.SCORE_GAP
+
+
 def test_step_and_score_with_many_short_rows(B):
     """70 000 trajectories of 8 elements: one CTA per row, more rows than a 16-bit grid dimension."""
     G, N0, d = 700, 100, 8
