@@ -67,10 +67,10 @@ def test_gpu_arm_prints_roofline_baseline_and_end_to_end():
     assert set(d["clocks"]) >= {"sm_mhz", "sm_max_mhz", "reasons"}
 
 
-def _torchrun(args, timeout=600):
+def _torchrun(args, timeout=600, port_offset=0):
     """One rank under the distributed launcher (rendezvous on 127.0.0.1): the process-group set-up,
     the build barrier, the max-over-ranks reduction and the gather all execute, on one GPU."""
-    port = 23000 + os.getpid() % 4000
+    port = 23000 + (os.getpid() % 4000) * 2 + port_offset      # a port of its own for every launch
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "1",
            "--master-addr", "127.0.0.1", "--master-port", str(port)] + args
     env = dict(os.environ, NCCL_NVLS_ENABLE="0")
@@ -94,7 +94,7 @@ def test_gpu_arm_under_the_distributed_launcher():
 @pytest.mark.gpu
 def test_sharded_launcher_runs_and_gathers():
     lines = _torchrun(["-m", "paper_2512_15347_b200.sharded", "--workload", "sd15", "--groups", "5",
-                       "--reps", "2"])
+                       "--reps", "2"], port_offset=1)
     assert len(lines) == 1
     d = json.loads(lines[0])
     assert d["ranks"] == 1 and d["groups"] == 5 and d["shards"] == [[0, 5]] and d["survivors"] == 5 * 12
