@@ -146,27 +146,38 @@ __device__ __forceinline__ double warp_sum(double v) {
 
 // ---------------------------------------------------------------- launch geometry
 // Row-streaming kernels (step, score, policy log-prob): a CTA of kRowThreads threads handles one
-// chunk of one row and contributes one partial sum, so a row owns `chunks` partial slots.  A chunk
-// is 2048 quads (4-element groups) whatever the number of rows, so the shape of a row's reduction
-// depends on the row length alone: a trajectory gets the same bits in a batch of any size, on any
-// shard.  Measured on 192 ... 4096 rows of 65536 quads, back-to-back launches: 1024-quad chunks
-// are 10 % slower (a CTA's launch, its first unoverlapped loads and its end-of-CTA barrier, fence
-// and atomic come twice as often), 3072- and 4096-quad chunks 1 - 3 % slower (fewer, longer CTAs
-// drain less evenly at the end of a launch).
+// chunk of one row and contributes one partial sum, so a row owns `chunks` partial slots.  Chunks
+// are 2048 or 4096 quads (4-element groups): the longer one wherever it still leaves about 16
+// waves of CTAs.  Measured under sustained load (60 rollouts of the large workload's launch mix
+// back to back, the board at its power cap): 4096-quad chunks 16.31 ms, 2048-quad chunks 16.60 ms,
+// 8192-quad chunks 16.68 ms per 28 launches of 4096 / 2048 / 1024 rows; on launches of 768 / 384 /
+// 192 rows 2048-quad chunks 3.25 ms against 3.28 ms (fewer, longer CTAs drain less evenly at the
+// end of a short launch).  In bursts of a few dozen launches, before the power cap bites, 2048-quad
+// chunks are 1 % faster at every size: a CTA's prologue and end-of-CTA reduction cost instructions,
+// and instructions cost clock once the board is power-limited.
 constexpr int kRowThreads = 256;
 constexpr int kRowWarps = kRowThreads / 32;
-constexpr int kChunkQuads = 2048;                      // 8192 elements per CTA
+constexpr int kMinChunkQuads = 2048;                   // 8192 elements
+constexpr int kMaxChunkQuads = 4096;                   // 16384 elements
+constexpr long long kWantedCtas = 148LL * 4 * 16;      // CTAs for ~16 waves at 4 CTAs per SM
 
 struct RowGeometry {
   int chunk_quads;   // quads per CTA
   int chunks;        // CTAs per row = partial sums per row
 };
 
-inline RowGeometry row_geometry(long long /*rows*/, int elems, int forced_chunk_quads = 0) {
+// Longest chunk that still leaves kWantedCtas CTAs, but never shorter than kMinChunkQuads.
+inline RowGeometry row_geometry(long long rows, int elems, int forced_chunk_quads = 0) {
   const int quads = elems / 4;
+  int cq = kMaxChunkQuads;
+  if (forced_chunk_quads > 0) {
+    cq = forced_chunk_quads;
+  } else {
+    while (cq > kMinChunkQuads && rows * ((quads + cq - 1) / cq) < kWantedCtas) cq >>= 1;
+  }
   RowGeometry g;
-  g.chunk_quads = forced_chunk_quads > 0 ? forced_chunk_quads : kChunkQuads;
-  g.chunks = (quads + g.chunk_quads - 1) / g.chunk_quads;
+  g.chunk_quads = cq;
+  g.chunks = (quads + cq - 1) / cq;
   return g;
 }
 

@@ -71,7 +71,7 @@ template <typename VelT, bool kNoise, bool kMean> struct StepMinCtas {
   static constexpr int value = (sizeof(VelT) == 2 && kNoise && !kMean) ? PG_STEP_MIN_CTAS : 4;
 };
 constexpr int kStepUnroll = PG_STEP_UNROLL;
-static_assert(kChunkQuads % (2 * kStepUnroll * kRowThreads) == 0,
+static_assert(kMinChunkQuads % (2 * kStepUnroll * kRowThreads) == 0 && kMaxChunkQuads % kMinChunkQuads == 0,
               "full chunks must hold an even number of batches");
 
 // One quad: mean of the transition, noise, store, radius-term accumulation.
